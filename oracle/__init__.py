@@ -1,0 +1,141 @@
+"""ctypes binding of the CPU oracle (oracle/ga_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the CPU-baseline leg
+of the benchmark. The CUDA library never imports or links this package.
+"""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ga_oracle.cpp")
+_LIB = os.path.join(_HERE, "libga_oracle.so")
+
+ASGD, SA, GA = 0, 1, 2
+CXXFLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-Wall", "-Wextra"]
+
+
+def build(force=False, src=_SRC, out=_LIB):
+    """Compile the oracle with g++ (no fast-math, no FMA contraction)."""
+    if not force and os.path.exists(out) and os.path.getmtime(out) >= os.path.getmtime(src):
+        return out
+    subprocess.check_call(["g++", *CXXFLAGS, "-o", out, src])
+    return out
+
+
+def _bind(path):
+    lib = ctypes.CDLL(path)
+    c = ctypes
+    lib.gao_create.restype = c.c_void_p
+    lib.gao_create.argtypes = [c.c_int64, c.c_int, c.c_double, c.c_double, c.c_double, c.c_int, c.c_int]
+    lib.gao_destroy.argtypes = [c.c_void_p]
+    lib.gao_set_c_order.argtypes = [c.c_void_p, c.c_int]
+    lib.gao_set_eps.argtypes = [c.c_void_p, c.c_double]
+    lib.gao_set_params.argtypes = [c.c_void_p, c.c_void_p]
+    lib.gao_pull.argtypes = [c.c_void_p, c.c_int]
+    lib.gao_push.restype = c.c_int64
+    lib.gao_push.argtypes = [c.c_void_p, c.c_int, c.c_void_p]
+    lib.gao_gap.argtypes = [c.c_void_p, c.c_int, c.c_void_p]
+    lib.gao_k_done.restype = c.c_int64
+    lib.gao_k_done.argtypes = [c.c_void_p]
+    lib.gao_iter.restype = c.c_int64
+    lib.gao_iter.argtypes = [c.c_void_p, c.c_int]
+    lib.gao_stats.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.gao_get.restype = c.c_int
+    lib.gao_get.argtypes = [c.c_void_p, c.c_int, c.c_void_p]
+    lib.gao_sent_f32.argtypes = [c.c_void_p, c.c_int, c.c_void_p]
+    return lib
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = _bind(build())
+    return _lib
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a
+
+
+class Oracle:
+    """One simulated master. precision=32 computes in fp32 (the parity reference for the
+    fp32 CUDA path); precision=64 runs the same steps in fp64."""
+
+    THETA, V, M, C = 0, 1, 2, 3
+
+    def __init__(self, n_params, n_workers, lr, momentum, c_beta, variant, precision=32,
+                 c_order=0, eps=None, _lib=None):
+        self._l = _lib if _lib is not None else lib()
+        self.d, self.n = int(n_params), int(n_workers)
+        self._h = self._l.gao_create(self.d, self.n, lr, momentum, c_beta, variant, precision)
+        if not self._h:
+            raise ValueError("gao_create failed")
+        self._l.gao_set_c_order(self._h, c_order)
+        if eps is not None:
+            self._l.gao_set_eps(self._h, eps)
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            self._l.gao_destroy(self._h)
+            self._h = None
+
+    def set_params(self, theta0):
+        a = _f32(theta0)
+        assert a.shape == (self.d,)
+        self._l.gao_set_params(self._h, a.ctypes.data)
+
+    def pull(self, worker):
+        assert 0 <= worker < self.n
+        self._l.gao_pull(self._h, worker)
+
+    def push(self, worker, grad):
+        assert 0 <= worker < self.n
+        g = _f32(grad)
+        assert g.shape == (self.d,)
+        return int(self._l.gao_push(self._h, worker, g.ctypes.data))
+
+    def push_batch(self, schedule, grads):
+        """push(i, g) then pull(i) for each arrival, in order. Returns the delays."""
+        delays = []
+        for i, g in zip(schedule, grads):
+            delays.append(self.push(i, g))
+            self.pull(i)
+        return delays
+
+    def get(self, which):
+        out = np.empty(self.d, dtype=np.float64)
+        rc = self._l.gao_get(self._h, which, out.ctypes.data)
+        assert rc == 0
+        return out
+
+    def saved(self, worker):
+        return self.get(4 + worker)
+
+    def sent_f32(self, worker):
+        out = np.empty(self.d, dtype=np.float32)
+        self._l.gao_sent_f32(self._h, worker, out.ctypes.data)
+        return out
+
+    def gap(self, worker):
+        out = np.empty(self.d, dtype=np.float64)
+        self._l.gao_gap(self._h, worker, out.ctypes.data)
+        return out
+
+    def stats(self):
+        s, m = ctypes.c_double(), ctypes.c_double()
+        self._l.gao_stats(self._h, ctypes.byref(s), ctypes.byref(m))
+        return s.value, m.value
+
+    @property
+    def k_done(self):
+        return int(self._l.gao_k_done(self._h))
+
+    def iter(self, worker):
+        return int(self._l.gao_iter(self._h, worker))

@@ -1,0 +1,274 @@
+// Reference ("oracle") implementation of the parameter-server update of Gap-Aware
+// asynchronous SGD (arXiv 1909.10802), with Staleness-Aware and plain momentum-ASGD
+// as variants.
+//
+// THIS IS TEST INFRASTRUCTURE. It is a plain, single-threaded, obviously-correct CPU
+// program that follows the paper's algorithms step by step. Only the tests, the smoke
+// check and the CPU-baseline leg of the benchmark may use it. It shares no code with
+// the CUDA library and neither includes the other.
+//
+// What follows which passage of the paper:
+//   push, variant ASGD : Algorithm "Momentum-ASGD: master" (Section 4)
+//   push, variant SA   : Algorithm "Staleness-Aware: master" (Section 4.1)
+//   push, variant GA   : Algorithm "Gap-Aware: master" (Section 5) with the
+//                        parameter-wise Gap of Section 5.3 (|theta_k - theta_{k-tau}|/C + 1)
+//   C                  : Algorithm "C Coefficient Calculation" (Appendix, C Coefficient)
+//   pull               : "Send theta_{k+1} to worker i" / "Save and send current
+//                        parameters" of the three master algorithms; the saved copy is
+//                        the theta^i = theta_{k-tau_k} of the appendix's remark
+//   momentum           : Section 3, the variant without dampening: v <- gamma v + g
+//
+// Readings taken where the paper leaves a choice (all also listed in the design notes):
+//   * Order of C and Gap (option c_order). 0 = "lagged": the Gap at arrival k uses the C
+//     that stands after arrival k-1; after the step, the second moment m is refreshed with
+//     the update vector actually applied (the master's new v). 1 = "Adam order": first
+//     u = gamma v + g with the raw gradient (the printed line of the C algorithm),
+//     m <- beta m + (1-beta) u^2, C from the new m, then Gap, penalised gradient, v, theta.
+//   * "Initialize C <- 0": before any refresh, C = eta_max * eps (the last line of the C
+//     algorithm at m_hat = 0), so the first Gap is 0/C + 1 = 1, not 0/0.
+//   * The exponent of the bias correction is the number of refreshes of m so far.
+//   * eps = 1e-8 is added after the square root, inside the eta_max product.
+//   * eta_max is the learning rate given at creation.
+//   * delay tau_k = k - iter[i], k counting arrivals from 1, iter[] starting at 0;
+//     a pull records the number of pushes applied so far.
+//   * Arithmetic: every line below is one IEEE operation per symbol, in the order
+//     written, with v <- gamma*v + g_hat and theta <- theta - eta*v each a single fused
+//     multiply-add. Build with -ffp-contract=off so nothing else is fused.
+//
+// Parity pins (tests/test_oracle_pins.py): Gap >= 1 and Gap == 1 where the saved copy
+// equals the master; one worker reduces to heavy-ball SGD (closed form); the SA two-step
+// expansion of Section 4.1; gamma = 0; constant |v| gives C = eta_max (c + eps) at every k;
+// same-direction steps give Gap = tau; round-robin delays; an exact-rational brute force.
+// "parity unpinned": the choice between the two c_order readings and the value of C
+// before the first refresh -- nothing the paper prints separates them.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+enum Variant { ASGD = 0, SA = 1, GA = 2 };
+
+template <typename T>
+struct Master {
+    int64_t d = 0;
+    int n_workers = 0;
+    T eta = 0;        // learning rate eta_k (constant here)
+    T eta_max = 0;    // eta_max of the C algorithm
+    T gamma = 0;      // momentum
+    T beta = 0;       // beta_1 of the C algorithm
+    T eps = (T)1e-8;  // epsilon of the C algorithm
+    int variant = GA;
+    int c_order = 0;  // 0 lagged, 1 Adam order
+    std::vector<T> theta, v, m;
+    std::vector<T> saved;       // N x d, row i = theta^i, the parameters last sent to worker i
+    std::vector<int64_t> iter;  // iteration array of the SA algorithm
+    int64_t k_done = 0;         // arrivals applied so far
+    int64_t k_c = 0;            // refreshes of m so far
+    double last_sum_gap = 0.0, last_max_gap = 0.0;
+
+    // 1 / (1 - beta^k) of the bias correction, k = refreshes of m so far (k >= 1).
+    T inv_bias() const { return (T)(1.0 / (1.0 - std::pow((double)beta, (double)k_c))); }
+
+    // C from the second moment as it stands (C algorithm, last two lines).
+    T coeff(T m_j, T inv_bias_k) const {
+        if (k_c == 0) return eta_max * eps;
+        const T m_hat = m_j * inv_bias_k;
+        return eta_max * (std::sqrt(m_hat) + eps);
+    }
+
+    void set_params(const float* theta0) {
+        for (int64_t j = 0; j < d; ++j) {
+            theta[j] = (T)theta0[j];
+            v[j] = 0;
+            m[j] = 0;
+        }
+        for (int i = 0; i < n_workers; ++i)
+            for (int64_t j = 0; j < d; ++j) saved[(size_t)i * d + j] = theta[j];
+        for (int i = 0; i < n_workers; ++i) iter[i] = 0;
+        k_done = 0;
+        k_c = 0;
+    }
+
+    void pull(int i) {
+        for (int64_t j = 0; j < d; ++j) saved[(size_t)i * d + j] = theta[j];
+        iter[i] = k_done;
+    }
+
+    int64_t push(int i, const float* grad) {
+        const int64_t k = k_done + 1;
+        const int64_t tau = k - iter[i];
+        const T* s = &saved[(size_t)i * d];
+        if (variant == ASGD) {
+            for (int64_t j = 0; j < d; ++j) {
+                const T g = (T)grad[j];
+                v[j] = std::fma(gamma, v[j], g);
+                theta[j] = std::fma(-eta, v[j], theta[j]);
+            }
+        } else if (variant == SA) {
+            const T eta_tau = eta / (T)tau;
+            for (int64_t j = 0; j < d; ++j) {
+                const T g = (T)grad[j];
+                v[j] = std::fma(gamma, v[j], g);
+                theta[j] = std::fma(-eta_tau, v[j], theta[j]);
+            }
+        } else {
+            const T one_minus_beta = (T)(1.0 - (double)beta);
+            double sum_gap = 0.0, max_gap = 0.0;
+            if (c_order == 1) {
+                // Adam order: refresh m from u = gamma v + g (raw gradient) first.
+                for (int64_t j = 0; j < d; ++j) {
+                    const T u = std::fma(gamma, v[j], (T)grad[j]);
+                    m[j] = std::fma(beta, m[j], one_minus_beta * (u * u));
+                }
+                k_c += 1;
+            }
+            const T ib = k_c > 0 ? inv_bias() : (T)0;
+            for (int64_t j = 0; j < d; ++j) {
+                const T g = (T)grad[j];
+                const T C = coeff(m[j], ib);
+                const T dist = std::fabs(theta[j] - s[j]);
+                const T G = dist / C + (T)1;
+                const T g_hat = g / G;
+                v[j] = std::fma(gamma, v[j], g_hat);
+                theta[j] = std::fma(-eta, v[j], theta[j]);
+                sum_gap += (double)G;
+                if ((double)G > max_gap) max_gap = (double)G;
+            }
+            if (c_order == 0) {
+                for (int64_t j = 0; j < d; ++j)
+                    m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));
+                k_c += 1;
+            }
+            last_sum_gap = sum_gap;
+            last_max_gap = max_gap;
+        }
+        k_done = k;
+        return tau;
+    }
+
+    // Gap of worker i against the master as it stands; changes nothing.
+    void gap(int i, double* out) const {
+        const T* s = &saved[(size_t)i * d];
+        const T ib = k_c > 0 ? inv_bias() : (T)0;
+        for (int64_t j = 0; j < d; ++j) {
+            const T C = coeff(m[j], ib);
+            const T dist = std::fabs(theta[j] - s[j]);
+            out[j] = (double)(dist / C + (T)1);
+        }
+    }
+};
+
+struct Handle {
+    int precision;  // 32 or 64
+    Master<float>* f;
+    Master<double>* g;
+};
+
+template <typename T>
+Master<T>* make(int64_t d, int n, double lr, double momentum, double beta, int variant) {
+    auto* M = new Master<T>();
+    M->d = d;
+    M->n_workers = n;
+    // Hyper-parameters arrive as fp32 values (the library's interface takes floats).
+    M->eta = (T)(float)lr;
+    M->eta_max = (T)(float)lr;
+    M->gamma = (T)(float)momentum;
+    M->beta = (T)(float)beta;
+    M->variant = variant;
+    M->theta.assign(d, 0);
+    M->v.assign(d, 0);
+    M->m.assign(d, 0);
+    M->saved.assign((size_t)n * d, 0);
+    M->iter.assign(n, 0);
+    return M;
+}
+
+}  // namespace
+
+#define DISPATCH(h, call) ((h)->precision == 32 ? (h)->f->call : (h)->g->call)
+
+extern "C" {
+
+void* gao_create(int64_t d, int n_workers, double lr, double momentum, double beta, int variant,
+                 int precision) {
+    if (d <= 0 || n_workers <= 0 || (precision != 32 && precision != 64)) return nullptr;
+    if (variant < 0 || variant > 2) return nullptr;
+    auto* h = new (std::nothrow) Handle{precision, nullptr, nullptr};
+    if (!h) return nullptr;
+    try {
+        if (precision == 32) h->f = make<float>(d, n_workers, lr, momentum, beta, variant);
+        else h->g = make<double>(d, n_workers, lr, momentum, beta, variant);
+    } catch (...) {
+        delete h;
+        return nullptr;
+    }
+    return h;
+}
+
+void gao_destroy(void* p) {
+    auto* h = (Handle*)p;
+    if (!h) return;
+    delete h->f;
+    delete h->g;
+    delete h;
+}
+
+void gao_set_c_order(void* p, int c_order) {
+    auto* h = (Handle*)p;
+    if (h->precision == 32) h->f->c_order = c_order; else h->g->c_order = c_order;
+}
+
+void gao_set_eps(void* p, double eps) {
+    auto* h = (Handle*)p;
+    if (h->precision == 32) h->f->eps = (float)eps; else h->g->eps = eps;
+}
+
+void gao_set_params(void* p, const float* theta0) { auto* h = (Handle*)p; DISPATCH(h, set_params(theta0)); }
+void gao_pull(void* p, int worker) { auto* h = (Handle*)p; DISPATCH(h, pull(worker)); }
+int64_t gao_push(void* p, int worker, const float* grad) { auto* h = (Handle*)p; return DISPATCH(h, push(worker, grad)); }
+void gao_gap(void* p, int worker, double* out) { auto* h = (Handle*)p; DISPATCH(h, gap(worker, out)); }
+int64_t gao_k_done(void* p) { auto* h = (Handle*)p; return h->precision == 32 ? h->f->k_done : h->g->k_done; }
+int64_t gao_iter(void* p, int worker) { auto* h = (Handle*)p; return h->precision == 32 ? h->f->iter[worker] : h->g->iter[worker]; }
+
+void gao_stats(void* p, double* sum_gap, double* max_gap) {
+    auto* h = (Handle*)p;
+    *sum_gap = h->precision == 32 ? h->f->last_sum_gap : h->g->last_sum_gap;
+    *max_gap = h->precision == 32 ? h->f->last_max_gap : h->g->last_max_gap;
+}
+
+// which: 0 theta, 1 v, 2 m, 3 C (derived from m), 4+i saved copy of worker i. Output in double.
+int gao_get(void* p, int which, double* out) {
+    auto* h = (Handle*)p;
+    auto copy = [&](auto* M) -> int {
+        const int64_t d = M->d;
+        if (which == 0) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->theta[j];
+        else if (which == 1) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->v[j];
+        else if (which == 2) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->m[j];
+        else if (which == 3) {
+            const auto ib = M->k_c > 0 ? M->inv_bias() : 0;
+            for (int64_t j = 0; j < d; ++j) out[j] = (double)M->coeff(M->m[j], ib);
+        }
+        else if (which >= 4 && which < 4 + M->n_workers)
+            for (int64_t j = 0; j < d; ++j) out[j] = (double)M->saved[(size_t)(which - 4) * d + j];
+        else return -1;
+        return 0;
+    };
+    return h->precision == 32 ? copy(h->f) : copy(h->g);
+}
+
+// The saved copy of one worker rounded to fp32: what is "sent" to the worker.
+void gao_sent_f32(void* p, int worker, float* out) {
+    auto* h = (Handle*)p;
+    if (h->precision == 32) {
+        std::memcpy(out, &h->f->saved[(size_t)worker * h->f->d], sizeof(float) * h->f->d);
+    } else {
+        const double* s = &h->g->saved[(size_t)worker * h->g->d];
+        for (int64_t j = 0; j < h->g->d; ++j) out[j] = (float)s[j];
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,395 @@
+"""Pins that tie the CPU oracle to what the paper and the mathematics fix.
+
+Each pin takes `make`, a factory with the signature of oracle.Oracle, so the same checks can
+be run against a deliberately broken build of the oracle (tests/test_oracle_mutants.py).
+Nothing here restates the oracle's loop: a pin is a closed form, an invariant, a special case
+that collapses to a textbook routine, a hand-worked value, or an exact-arithmetic brute force.
+"""
+import os
+from decimal import Decimal, getcontext
+from fractions import Fraction
+
+import numpy as np
+
+ASGD, SA, GA = 0, 1, 2
+THETA, V, M, C = 0, 1, 2, 3
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+def _f32(x):
+    return np.asarray(x, dtype=np.float32)
+
+
+# --------------------------------------------------------------------------------------
+def pin_gap_is_one_where_copy_equals_master(make):
+    """Definition 1 / Section 4.1 'Over-Penalizing': where theta_k equals the saved copy the
+    Gap is exactly 1 and the gradient goes through unpenalised, while SA still divides by tau."""
+    d, eta = 64, 0.1
+    r = _rng(1)
+    th0 = _f32(r.normal(size=d))
+    g1 = _f32(r.normal(size=d))
+    g1[1::2] = 0.0                      # worker 1 moves only the even elements
+    g0 = _f32(r.normal(size=d))
+    res = {}
+    for variant in (GA, ASGD, SA):
+        o = make(d, 2, eta, 0.9, 0.999, variant, precision=32)
+        o.set_params(th0)
+        assert o.push(1, g1) == 1
+        o.pull(1)
+        if variant == GA:
+            G = o.gap(0)
+            assert np.all(G >= 1.0)
+            assert np.all(G[1::2] == 1.0), "Gap must be exactly 1 where the copy equals the master"
+            assert np.all(G[0::2][g1[0::2] != 0] > 1.0)
+        assert o.push(0, g0) == 2       # delay 2 although the odd elements never moved
+        res[variant] = (o.get(THETA), o.get(V))
+    odd = slice(1, None, 2)
+    # GA == unpenalised momentum step, bit for bit, on the untouched elements ...
+    assert np.array_equal(res[GA][0][odd], res[ASGD][0][odd])
+    assert np.array_equal(res[GA][1][odd], res[ASGD][1][odd])
+    # ... and that step is theta0 - eta*g0 (v was 0 there)
+    want = th0.astype(np.float64)[odd] - np.float64(np.float32(eta)) * g0.astype(np.float64)[odd]
+    assert np.allclose(res[GA][0][odd], want, rtol=0, atol=2e-7)
+    # SA halves the step there (tau = 2): over-penalised
+    want_sa = th0.astype(np.float64)[odd] - np.float64(np.float32(eta)) / 2 * g0.astype(np.float64)[odd]
+    assert np.allclose(res[SA][0][odd], want_sa, rtol=0, atol=2e-7)
+    # on the moved elements GA penalises: |step| strictly smaller than the unpenalised one
+    ev = slice(0, None, 2)
+    moved = g1[ev] != 0
+    v_prev = g1.astype(np.float64)[ev]
+    pen = np.abs(res[GA][1][ev] - 0.9 * v_prev)[moved]      # |g_hat|
+    raw = np.abs(res[ASGD][1][ev] - 0.9 * v_prev)[moved]    # |g|
+    assert np.all(pen < raw + 1e-12) and np.any(pen < 0.9 * raw)
+
+
+def pin_one_worker_is_heavy_ball(make):
+    """Section 3: with one worker (push, pull, push, ...) every delay is 1 and the saved copy is
+    always current, so GA, SA and ASGD are the momentum method without dampening -- checked
+    against torch.optim.SGD(momentum) and against the closed form for a constant gradient."""
+    import torch
+    d, eta, gam, steps = 33, 0.05, 0.9, 25
+    r = _rng(2)
+    th0 = _f32(r.normal(size=d))
+    grads = [_f32(r.normal(size=d)) for _ in range(steps)]
+    out = {}
+    for variant in (GA, SA, ASGD):
+        for prec in (32, 64):
+            o = make(d, 1, eta, gam, 0.999, variant, precision=prec)
+            o.set_params(th0)
+            for g in grads:
+                assert o.push(0, g) == 1
+                o.pull(0)
+            out[(variant, prec)] = (o.get(THETA), o.get(V))
+    for prec in (32, 64):
+        for variant in (GA, SA):
+            assert np.array_equal(out[(variant, prec)][0], out[(ASGD, prec)][0])
+            assert np.array_equal(out[(variant, prec)][1], out[(ASGD, prec)][1])
+    p = torch.tensor(th0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([p], lr=float(np.float32(eta)), momentum=float(np.float32(gam)), dampening=0.0)
+    for g in grads:
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+    assert np.allclose(out[(ASGD, 64)][0], p.detach().numpy(), rtol=1e-12, atol=1e-13)
+    assert np.allclose(out[(ASGD, 32)][0], p.detach().numpy(), rtol=1e-5, atol=1e-5)
+    # constant gradient c: v_k = c (1-gam^k)/(1-gam); theta_k = theta_0 - eta * sum_t v_t
+    c = _f32(r.normal(size=d))
+    o = make(d, 1, eta, gam, 0.999, ASGD, precision=64)
+    o.set_params(th0)
+    e, g_ = float(np.float32(eta)), float(np.float32(gam))
+    for k in range(1, 12):
+        o.push(0, c)
+        o.pull(0)
+        vk = c.astype(np.float64) * (1 - g_ ** k) / (1 - g_)
+        sk = c.astype(np.float64) * (k - g_ * (1 - g_ ** k) / (1 - g_)) / (1 - g_)
+        assert np.allclose(o.get(V), vk, rtol=1e-12, atol=1e-14)
+        assert np.allclose(o.get(THETA), th0.astype(np.float64) - e * sk, rtol=1e-12, atol=1e-13)
+
+
+def pin_sa_two_step_expansion(make):
+    """Section 4.1 'Under-Penalizing': theta_{k+2} = theta_{k+1} - (eta/tau_{k+1})
+    (gam^2 v_k + gam g_k + g_{k+1}), and theta_{k+1} = theta_k - (eta/tau_k)(gam v_k + g_k);
+    delays for the schedule 0,1,2,0,2 worked by hand: 1,2,3,3,2."""
+    d, eta, gam = 17, 0.1, 0.9
+    r = _rng(3)
+    th0 = _f32(r.normal(size=d))
+    sched, want_tau = [0, 1, 2, 0, 2], [1, 2, 3, 3, 2]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    o = make(d, 3, eta, gam, 0.999, SA, precision=64)
+    o.set_params(th0)
+    th, v = [o.get(THETA)], [o.get(V)]
+    taus = []
+    for i, g in zip(sched, grads):
+        taus.append(o.push(i, g))
+        o.pull(i)
+        th.append(o.get(THETA))
+        v.append(o.get(V))
+    assert taus == want_tau
+    e, g_ = float(np.float32(eta)), float(np.float32(gam))
+    G = [g.astype(np.float64) for g in grads]
+    for k in range(len(sched)):
+        one = th[k] - e / want_tau[k] * (g_ * v[k] + G[k])
+        assert np.allclose(th[k + 1], one, rtol=1e-13, atol=1e-14)
+    for k in range(len(sched) - 1):
+        two = th[k + 1] - e / want_tau[k + 1] * (g_ * g_ * v[k] + g_ * G[k] + G[k + 1])
+        assert np.allclose(th[k + 2], two, rtol=1e-13, atol=1e-14)
+    # and the fp32 build agrees to rounding
+    o32 = make(d, 3, eta, gam, 0.999, SA, precision=32)
+    o32.set_params(th0)
+    assert o32.push_batch(sched, grads) == want_tau
+    assert np.allclose(o32.get(THETA), th[-1], rtol=1e-5, atol=1e-6)
+
+
+def pin_zero_momentum(make):
+    """Section 6 'ASGD': gamma = 0 leaves theta <- theta - eta * g_hat and v = g_hat."""
+    d, eta = 21, 0.2
+    r = _rng(4)
+    th0 = _f32(r.normal(size=d))
+    o = make(d, 2, eta, 0.0, 0.999, ASGD, precision=64)
+    o.set_params(th0)
+    acc = th0.astype(np.float64)
+    for k in range(6):
+        g = _f32(r.normal(size=d))
+        o.push(k % 2, g)
+        o.pull(k % 2)
+        acc = acc - float(np.float32(eta)) * g.astype(np.float64)
+        assert np.array_equal(o.get(V), g.astype(np.float64))
+        assert np.allclose(o.get(THETA), acc, rtol=1e-14, atol=1e-15)
+    # SA with gamma = 0: plain SGD with the step divided by the delay
+    o = make(d, 3, eta, 0.0, 0.999, SA, precision=64)
+    o.set_params(th0)
+    acc = th0.astype(np.float64)
+    for k, (i, tau) in enumerate(zip([0, 1, 2, 1], [1, 2, 3, 2])):
+        g = _f32(r.normal(size=d))
+        assert o.push(i, g) == tau
+        o.pull(i)
+        acc = acc - float(np.float32(eta)) / tau * g.astype(np.float64)
+        assert np.allclose(o.get(THETA), acc, rtol=1e-14, atol=1e-15)
+
+
+def pin_constant_magnitude_gives_constant_C(make):
+    """C Coefficient algorithm: if |v| = c at every step, the bias-corrected second moment is
+    c^2 at every k, so C = eta_max (c + eps) from the first refresh on (the Adam-style
+    correction with exponent k = number of refreshes)."""
+    d, eta, beta, eps = 16, 0.1, 0.999, 1e-8
+    c = _f32(np.linspace(0.01, 3.0, d))
+    sign = np.ones(d, dtype=np.float32)
+    for c_order in (0, 1):
+        o = make(d, 1, eta, 0.0, beta, GA, precision=64, c_order=c_order)
+        o.set_params(np.zeros(d, np.float32))
+        want = float(np.float32(eta)) * (c.astype(np.float64) + eps)
+        for k in range(1, 40):
+            sign = -sign if k % 3 == 0 else sign
+            o.push(0, c * sign)
+            o.pull(0)
+            assert np.allclose(o.get(C), want, rtol=1e-11, atol=0), f"C drifted at k={k}"
+    # fp32 build: same to fp32 rounding
+    o = make(d, 1, eta, 0.0, beta, GA, precision=32)
+    o.set_params(np.zeros(d, np.float32))
+    for k in range(1, 40):
+        o.push(0, c)
+        o.pull(0)
+        assert np.allclose(o.get(C), want, rtol=3e-5, atol=0)
+
+
+def pin_first_refresh(make):
+    """C Coefficient algorithm at k = 1: m_hat = v^2, so C = eta_max (|v| + eps); before any
+    refresh C = eta_max * eps (the reading of 'Initialize C <- 0')."""
+    d, eta = 12, 0.25
+    r = _rng(6)
+    th0 = _f32(r.normal(size=d))
+    g = _f32(r.normal(size=d))
+    o = make(d, 2, eta, 0.9, 0.75, GA, precision=64)
+    o.set_params(th0)
+    assert np.allclose(o.get(C), 0.25 * 1e-8, rtol=1e-12)
+    assert np.array_equal(o.gap(0), np.ones(d))
+    o.push(0, g)
+    assert np.allclose(o.get(V), g.astype(np.float64), rtol=0, atol=0)
+    assert np.allclose(o.get(M), 0.25 * g.astype(np.float64) ** 2, rtol=1e-14)
+    assert np.allclose(o.get(C), 0.25 * (np.abs(g.astype(np.float64)) + 1e-8), rtol=1e-12)
+
+
+def pin_same_direction_steps_give_gap_tau(make):
+    """Section 5.1: E[G] = tau exactly when all tau updates went the same way. Worker B makes t
+    unpenalised steps of eta*c each (gamma = 0, its own copy always current) while worker A
+    holds theta_0: A's Gap is t + 1 = A's delay, and A's gradient is divided by it."""
+    d, eta, t = 8, 0.1, 6
+    c = _f32(np.linspace(0.5, 4.0, d))
+    o = make(d, 2, eta, 0.0, 0.999, GA, precision=64)
+    o.set_params(np.zeros(d, np.float32))
+    for k in range(t):
+        assert o.push(1, c) == (1 if k else 1)
+        o.pull(1)
+        assert np.array_equal(o.gap(1), np.ones(d))
+    e = float(np.float32(eta))
+    assert np.allclose(o.get(THETA), -t * e * c.astype(np.float64), rtol=1e-13)
+    G = o.gap(0)
+    assert np.allclose(G, t + 1, rtol=1e-6), G       # eps makes it a hair below t+1
+    assert np.all(G < t + 1) and np.all(G > t + 1 - 1e-5)
+    before = o.get(THETA)
+    assert o.push(0, c) == t + 1
+    assert np.allclose(o.get(V), c.astype(np.float64) / G, rtol=1e-13)
+    assert np.allclose(before - o.get(THETA), e * c.astype(np.float64) / G, rtol=1e-11)
+
+
+def pin_round_robin_delays(make):
+    """Staleness-Aware master: tau_k = k - iter[i]. N equal workers in round robin give
+    tau = k for the first N arrivals and N from then on ('tau scales linearly with N')."""
+    d, n = 4, 7
+    g = np.ones(d, np.float32)
+    for variant in (ASGD, SA, GA):
+        o = make(d, n, 0.01, 0.5, 0.999, variant, precision=32)
+        o.set_params(np.zeros(d, np.float32))
+        taus = o.push_batch([k % n for k in range(3 * n)], [g] * (3 * n))
+        assert taus == [k + 1 for k in range(n)] + [n] * (2 * n)
+        assert o.k_done == 3 * n
+    # a second push with no pull in between keeps measuring against the old copy
+    o = make(d, 2, 0.01, 0.5, 0.999, SA, precision=32)
+    o.set_params(np.zeros(d, np.float32))
+    assert [o.push(0, g), o.push(0, g), o.push(1, g), o.push(0, g)] == [1, 2, 3, 4]
+    o.pull(0)
+    assert o.iter(0) == 4 and o.push(0, g) == 1
+
+
+def pin_pull_saves_master(make):
+    """'Save and send current parameters': after pull(i) the saved copy of worker i is the
+    master's theta; other workers' copies are untouched; set_params seeds every copy."""
+    d = 9
+    r = _rng(8)
+    th0 = _f32(r.normal(size=d))
+    o = make(d, 3, 0.1, 0.9, 0.999, GA, precision=32)
+    o.set_params(th0)
+    for i in range(3):
+        assert np.array_equal(o.saved(i), th0.astype(np.float64))
+    o.push(0, _f32(r.normal(size=d)))
+    th1 = o.get(THETA)
+    assert not np.array_equal(th1, th0.astype(np.float64))
+    o.pull(2)
+    assert np.array_equal(o.saved(2), th1)
+    assert np.array_equal(o.saved(0), th0.astype(np.float64))
+    assert np.array_equal(o.saved(1), th0.astype(np.float64))
+    assert np.array_equal(o.sent_f32(2).astype(np.float64), th1)
+    # set_params starts a new run: v = m = 0, no arrivals counted, every copy = theta_0
+    o.set_params(th0)
+    assert not o.get(V).any() and not o.get(M).any() and o.k_done == 0 and o.iter(2) == 0
+    assert np.array_equal(o.saved(2), th0.astype(np.float64))
+
+
+def pin_hand_worked_example(make):
+    """Two arrivals worked by hand in exact fractions (tests/golden/ga_two_arrivals.txt)."""
+    vals = {}
+    with open(os.path.join(GOLDEN, "ga_two_arrivals.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = line.split("=")
+                vals[k.strip()] = Fraction(v.strip())
+    o = make(1, 2, float(vals["eta"]), float(vals["gamma"]), float(vals["beta"]), GA,
+             precision=64, eps=float(vals["eps"]))
+    o.set_params(_f32([float(vals["theta0"])]))
+    assert o.push(0, _f32([float(vals["g1"])])) == 1
+    o.pull(0)
+    for name, which in (("theta1", THETA), ("v1", V), ("m1", M), ("C1", C)):
+        assert abs(o.get(which)[0] - float(vals[name])) <= 1e-15 * max(1, abs(float(vals[name]))), name
+    assert abs(o.gap(1)[0] - float(vals["G2"])) < 1e-15 * 4
+    assert o.push(1, _f32([float(vals["g2"])])) == 2
+    for name, which in (("theta2", THETA), ("v2", V), ("m2", M)):
+        assert abs(o.get(which)[0] - float(vals[name])) <= 4e-16 * max(1, abs(float(vals[name]))), name
+    assert o.stats()[1] == o.stats()[0] and abs(o.stats()[0] - float(vals["G2"])) < 1e-15
+
+
+# ------------------------------------------------------------------ exact brute force
+def _sqrt_fraction(x):
+    getcontext().prec = 90
+    if x == 0:
+        return Fraction(0)
+    s = (Decimal(x.numerator) / Decimal(x.denominator)).sqrt()
+    return Fraction(s)
+
+
+def brute_force(th0, sched, grads, n, eta, gam, beta, eps, variant, c_order):
+    """The master algorithms of the paper in exact rational arithmetic (square roots to 90
+    digits), scalar by scalar. push followed by pull for each arrival."""
+    d = len(th0)
+    th = [Fraction(float(x)) for x in th0]
+    v = [Fraction(0)] * d
+    m = [Fraction(0)] * d
+    saved = [list(th) for _ in range(n)]
+    it = [0] * n
+    refreshes = 0
+    taus, gaps = [], []
+    for k, (i, g) in enumerate(zip(sched, grads), start=1):
+        g = [Fraction(float(x)) for x in g]
+        tau = k - it[i]
+        taus.append(tau)
+        for j in range(d):
+            if variant == ASGD:
+                v[j] = gam * v[j] + g[j]
+                th[j] = th[j] - eta * v[j]
+            elif variant == SA:
+                v[j] = gam * v[j] + g[j]
+                th[j] = th[j] - eta / tau * v[j]
+            else:
+                r = refreshes
+                mj = m[j]
+                if c_order == 1:
+                    u = gam * v[j] + g[j]
+                    mj = beta * mj + (1 - beta) * u * u
+                    r += 1
+                    m[j] = mj
+                Cj = eta * eps if r == 0 else eta * (_sqrt_fraction(mj / (1 - beta ** r)) + eps)
+                Gj = abs(th[j] - saved[i][j]) / Cj + 1
+                v[j] = gam * v[j] + g[j] / Gj
+                th[j] = th[j] - eta * v[j]
+                if c_order == 0:
+                    m[j] = beta * m[j] + (1 - beta) * v[j] * v[j]
+                if j == d - 1:
+                    gaps.append(Gj)
+        if variant == GA:
+            refreshes += 1
+        saved[i] = list(th)
+        it[i] = k
+    return th, v, m, taus
+
+
+def pin_exact_brute_force(make):
+    """Algorithms 'Momentum-ASGD', 'Staleness-Aware', 'Gap-Aware: master' and 'C Coefficient
+    Calculation' evaluated in exact arithmetic on d = 3, N = 3, 6 arrivals."""
+    r = _rng(10)
+    d, n = 3, 3
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 0, 2, 1, 0]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    eta, gam, beta, eps = 0.125, 0.75, 0.875, 1e-8      # dyadic: exact as fp32 and as fractions
+    F = Fraction
+    for variant in (ASGD, SA, GA):
+        for c_order in ((0, 1) if variant == GA else (0,)):
+            th, v, m, taus = brute_force(th0, sched, grads, n, F(eta), F(gam), F(beta), F(eps),
+                                         variant, c_order)
+            for prec, tol in ((64, 2e-13), (32, 2e-5)):
+                o = make(d, n, eta, gam, beta, variant, precision=prec, c_order=c_order, eps=eps)
+                o.set_params(th0)
+                assert o.push_batch(sched, grads) == taus
+                for which, ref in ((THETA, th), (V, v), (M, m)):
+                    got = o.get(which)
+                    want = np.array([float(x) for x in ref])
+                    assert np.all(np.abs(got - want) <= tol * (1 + np.abs(want))), \
+                        (variant, c_order, prec, which, got, want)
+
+
+ALL_PINS = [
+    pin_gap_is_one_where_copy_equals_master,
+    pin_one_worker_is_heavy_ball,
+    pin_sa_two_step_expansion,
+    pin_zero_momentum,
+    pin_constant_magnitude_gives_constant_C,
+    pin_first_refresh,
+    pin_same_direction_steps_give_gap_tau,
+    pin_round_robin_delays,
+    pin_pull_saves_master,
+    pin_hand_worked_example,
+    pin_exact_brute_force,
+]

@@ -1,0 +1,83 @@
+"""Each plausible mistake, planted in a copy of the oracle's source, must trip a pin.
+
+The mutants are textual edits of oracle/ga_oracle.cpp compiled into a temporary library; the
+committed oracle is never touched. A mutant that no pin catches means the pins are too weak.
+"""
+import os
+import subprocess
+
+import pytest
+
+import oracle
+from tests import oracle_pins
+
+SRC = os.path.join(os.path.dirname(oracle.__file__), "ga_oracle.cpp")
+
+# (name, text in the oracle, replacement)
+MUTANTS = [
+    ("gap_without_plus_one", "const T G = dist / C + (T)1;", "const T G = dist / C;"),
+    ("gap_multiplies_gradient", "const T g_hat = g / G;", "const T g_hat = g * G;"),
+    ("gap_divides_by_C_squared", "const T G = dist / C + (T)1;", "const T G = dist / C / C + (T)1;"),
+    ("gap_uses_signed_distance", "const T dist = std::fabs(theta[j] - s[j]);\n                const T G",
+     "const T dist = theta[j] - s[j];\n                const T G"),
+    ("gap_against_master_itself", "const T dist = std::fabs(theta[j] - s[j]);\n                const T G",
+     "const T dist = std::fabs(theta[j] - theta[j]);\n                const T G"),
+    ("momentum_with_dampening", "v[j] = std::fma(gamma, v[j], g_hat);",
+     "v[j] = std::fma(gamma, v[j], ((T)1 - gamma) * g_hat);"),
+    ("momentum_dropped_in_ga", "v[j] = std::fma(gamma, v[j], g_hat);", "v[j] = g_hat;"),
+    ("step_sign", "theta[j] = std::fma(-eta, v[j], theta[j]);\n                sum_gap",
+     "theta[j] = std::fma(eta, v[j], theta[j]);\n                sum_gap"),
+    ("step_uses_gradient_not_v", "theta[j] = std::fma(-eta, v[j], theta[j]);\n                sum_gap",
+     "theta[j] = std::fma(-eta, g_hat, theta[j]);\n                sum_gap"),
+    ("sa_multiplies_by_tau", "const T eta_tau = eta / (T)tau;", "const T eta_tau = eta * (T)tau;"),
+    ("sa_ignores_tau", "const T eta_tau = eta / (T)tau;", "const T eta_tau = eta;"),
+    ("sa_divides_gradient_twice", "const T eta_tau = eta / (T)tau;", "const T eta_tau = eta / (T)tau / (T)tau;"),
+    ("delay_off_by_one", "const int64_t tau = k - iter[i];", "const int64_t tau = k - iter[i] + 1;"),
+    ("delay_of_wrong_worker", "const int64_t tau = k - iter[i];", "const int64_t tau = k - iter[0];"),
+    ("pull_forgets_iteration", "iter[i] = k_done;\n", "\n"),
+    ("pull_saves_wrong_row", "saved[(size_t)i * d + j] = theta[j];\n        iter[i]",
+     "saved[(size_t)0 * d + j] = theta[j];\n        iter[i]"),
+    ("c_without_sqrt", "return eta_max * (std::sqrt(m_hat) + eps);", "return eta_max * (m_hat + eps);"),
+    ("c_without_eta_max", "return eta_max * (std::sqrt(m_hat) + eps);", "return (std::sqrt(m_hat) + eps);"),
+    ("c_eps_inside_sqrt", "return eta_max * (std::sqrt(m_hat) + eps);", "return eta_max * std::sqrt(m_hat + eps);"),
+    ("c_no_bias_correction", "const T m_hat = m_j * inv_bias_k;", "const T m_hat = m_j;"),
+    ("c_bias_exponent_off_by_one", "std::pow((double)beta, (double)k_c)", "std::pow((double)beta, (double)(k_c + 1))"),
+    ("c_bias_uses_beta_not_power", "std::pow((double)beta, (double)k_c)", "(double)beta"),
+    ("m_first_moment", "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));",
+     "m[j] = std::fma(beta, m[j], one_minus_beta * std::fabs(v[j]));"),
+    ("m_weights_swapped", "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));",
+     "m[j] = std::fma(one_minus_beta, m[j], beta * (v[j] * v[j]));"),
+    ("m_from_raw_gradient", "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));",
+     "m[j] = std::fma(beta, m[j], one_minus_beta * ((T)grad[j] * (T)grad[j]));"),
+    ("asgd_dampened", "v[j] = std::fma(gamma, v[j], g);\n                theta[j] = std::fma(-eta, v[j], theta[j]);",
+     "v[j] = std::fma(gamma, v[j], ((T)1 - gamma) * g);\n                theta[j] = std::fma(-eta, v[j], theta[j]);"),
+    ("adam_order_uses_penalised_v", "const T u = std::fma(gamma, v[j], (T)grad[j]);",
+     "const T u = v[j];"),
+    ("set_params_keeps_momentum", "v[j] = 0;\n            m[j] = 0;", "m[j] = 0;"),
+]
+
+
+def _build_mutant(tmp_path, name, old, new):
+    text = open(SRC).read()
+    assert text.count(old) >= 1, f"mutant {name}: target text not found in the oracle"
+    src = tmp_path / f"{name}.cpp"
+    src.write_text(text.replace(old, new, 1))
+    out = tmp_path / f"lib_{name}.so"
+    subprocess.check_call(["g++", *oracle.CXXFLAGS, "-w", "-o", str(out), str(src)])
+    return oracle._bind(str(out))
+
+
+@pytest.mark.parametrize("name,old,new", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_mutant_is_caught(tmp_path, name, old, new):
+    lib = _build_mutant(tmp_path, name, old, new)
+
+    def make(*a, **kw):
+        return oracle.Oracle(*a, _lib=lib, **kw)
+
+    caught = []
+    for pin in oracle_pins.ALL_PINS:
+        try:
+            pin(make)
+        except AssertionError:
+            caught.append(pin.__name__)
+    assert caught, f"no pin notices the mistake '{name}'"

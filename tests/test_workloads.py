@@ -1,0 +1,130 @@
+"""Synthetic-input generators: hash, shapes, schedules, gradients (CPU side)."""
+import numpy as np
+
+import workloads as W
+
+
+def test_splitmix64_published_outputs():
+    # word(key, b) is output b of SplitMix64 seeded with `key`; these are the generator's
+    # widely published first outputs for seed 1234567.
+    assert [W.word(1234567, b) for b in range(5)] == [
+        6457827717110365317, 3203168211198807973, 9817491932198370423,
+        4593380528125082431, 16408922859458223821]
+
+
+def test_c_and_python_hash_agree():
+    lib = W.cpu_lib()
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        seed, tag, a, b = (int(x) for x in rng.integers(0, 2**63, size=4))
+        assert lib.wl_cpu_hash(seed, tag % 8, a, b) == W.hash4(seed, tag % 8, a, b)
+        assert lib.wl_cpu_mix64(seed) == W.mix64(seed)
+
+
+def test_uniform_and_noise_fields():
+    lib = W.cpu_lib()
+    assert lib.wl_cpu_uniform(0) == np.float32(2.0 ** -24)
+    assert lib.wl_cpu_uniform(2**64 - 1) == np.float32(1.0 - 2.0 ** -24)
+    scale = np.float32(np.sqrt(3.0) / 65536)
+    assert lib.wl_cpu_xi(0) == np.float32(-131070) * scale
+    assert lib.wl_cpu_xi(2**64 - 1) == np.float32(131070) * scale
+    assert lib.wl_cpu_xi(0x0001_0002_0003_0004) == np.float32(10 - 131070) * scale
+
+
+def test_shapes_match_the_models():
+    assert (len(W.resnet20_segments()), sum(W.resnet20_segments())) == (65, 272_474)
+    assert (len(W.resnet50_segments()), sum(W.resnet50_segments())) == (161, 25_557_032)
+    assert sum(W.wrn16_4_segments()) == 2_748_890
+    seg = W.transformer_lm_segments()
+    assert seg[0] == 267_735 * 512 and sum(seg) == 150_000_000 and len(seg) == 17
+    for name, n, arrivals in (("C1", 8, 1000), ("C2", 32, 20000), ("C3", 64, 2000),
+                              ("C4", 128, 50000), ("C5", 32, 500)):
+        w = W.config(name)
+        assert (w.n_workers, w.arrivals) == (n, arrivals)
+
+
+def test_static_vectors_have_the_stated_distributions():
+    w = W.config("C1")
+    a, ts, t0 = w.curvature(), w.theta_star(), w.theta0()
+    assert 0.5 <= a.min() and a.max() <= 2.0 and abs(a.mean() - 1.25) < 0.01
+    assert abs(ts.std() - 0.1) < 2e-3 and abs(ts.mean()) < 1e-3
+    assert abs(t0.std() - 0.05) < 1e-3 and abs(t0.mean()) < 1e-3
+    idx = w.sample_indices(500)
+    assert np.array_equal(w.theta0(idx), t0[idx])
+    assert np.array_equal(w.curvature(idx), a[idx])
+
+
+def test_gradient_is_the_quadratic_model():
+    w = W.config("C1")
+    sent = w.theta0()
+    g = w.grad(7, sent)
+    a, ts = w.curvature().astype(np.float64), w.theta_star().astype(np.float64)
+    noise = g.astype(np.float64) - a * (sent.astype(np.float64) - ts)
+    assert abs(noise.std() - 0.01) < 2e-4 and abs(noise.mean()) < 1e-4
+    # another arrival draws other noise; sampled indices reproduce the dense values
+    assert not np.array_equal(w.grad(8, sent), g)
+    idx = w.sample_indices(777)
+    assert np.array_equal(w.grad(7, sent[idx], idx), g[idx])
+    # gradient at the minimiser is noise only
+    g_star = w.grad(7, w.theta_star())
+    assert abs(g_star.std() - 0.01) < 2e-4
+
+
+def test_per_segment_noise_scale():
+    w = W.config("mini")
+    assert w.seg_sigma.min() >= 1e-3 and w.seg_sigma.max() <= 1e-1
+    g = w.grad(3, w.theta_star()).astype(np.float64)
+    for l in (0, 2):
+        lo, hi = w.seg_off[l], w.seg_off[l + 1]
+        assert abs(g[lo:hi].std() / w.seg_sigma[l] - 1) < 0.1
+
+
+def test_sparse_embedding_rows():
+    w = W.config("C5")
+    rows = np.arange(0, 20000, dtype=np.int64)
+    idx = rows * 512 + 5
+    g1 = w.grad(1, np.zeros(len(idx), np.float32), idx)
+    active = g1 != 0
+    assert abs(active.mean() - 0.1) < 0.01
+    # a whole row shares its activity
+    idx2 = rows * 512 + 300
+    g2 = w.grad(1, np.zeros(len(idx), np.float32), idx2)
+    assert np.array_equal(g2 != 0, active)
+    # other arrival, other rows
+    g3 = w.grad(2, np.zeros(len(idx), np.float32), idx)
+    assert not np.array_equal(g3 != 0, active)
+    # dense region: never exactly sparse, std 0.01; independent of the sent parameters
+    tail = np.arange(w.d - 50000, w.d, dtype=np.int64)
+    gt = w.grad(1, np.zeros(len(tail), np.float32), tail)
+    assert abs(gt.std() - 0.01) < 3e-4 and (gt == 0).mean() < 1e-3
+    assert np.array_equal(gt, w.grad(1, np.ones(len(tail), np.float32), tail))
+
+
+def test_schedules():
+    for name in ("C1", "C2", "C4"):
+        w = W.config(name)
+        s = w.schedule()
+        assert len(s) == w.arrivals and set(s) <= set(range(w.n_workers))
+        assert len(set(s)) == w.n_workers, "every worker arrives at least once"
+        assert s == W.config(name).schedule(), "deterministic"
+    # equal speeds with 1..3 tick jitter: nobody laps anybody by much
+    s = W.config("C1").schedule()
+    counts = np.bincount(s, minlength=8)
+    assert counts.max() - counts.min() < 0.2 * counts.mean()
+    # stragglers: the 13 slow workers of C4 arrive about 5x less often
+    s = W.config("C4").schedule()
+    counts = np.sort(np.bincount(s, minlength=128))
+    assert 3.5 < counts[13:].mean() / counts[:13].mean() < 7
+    # log-normal: constant per-worker speed => strictly periodic arrivals of each worker
+    s = np.asarray(W.config("C2").schedule())
+    assert np.bincount(s).max() / np.bincount(s).min() > 2
+    assert W.schedule_round_robin(3, 7) == [0, 1, 2, 0, 1, 2, 0]
+
+
+def test_windows_never_repeat_a_worker():
+    s = W.config("C2").schedule()[:3000]
+    for k_max in (1, 4, 16):
+        ws = W.windows(s, k_max)
+        assert [i for w in ws for i in w] == s
+        assert all(len(w) <= k_max and len(set(w)) == len(w) for w in ws)
+    assert W.windows([0, 1, 0, 0, 2], 16) == [[0, 1], [0], [0, 2]]
