@@ -1,0 +1,158 @@
+/* ga.h -- C ABI of the Gap-Aware parameter-server ("master") update for NVIDIA B200.
+ *
+ * The library plays the master of asynchronous SGD with a parameter server
+ * (arXiv 1909.10802, Section 4): it owns the master parameters theta, the momentum (update
+ * vector) v, the running second moment m from which the coefficient C is derived, and one
+ * saved copy of the parameters per worker (theta^i, "the parameters last sent to worker i").
+ * Each arriving gradient is applied by one fused CUDA kernel; several consecutive arrivals
+ * can be applied by a single launch that keeps theta, v and m in registers.
+ *
+ * Conventions
+ *   - fp32 throughout. Pointers named *_dev are DEVICE pointers, 16-byte aligned, to at least
+ *     n_params floats; pointers named *_host are HOST pointers. The library owns theta, v, m
+ *     and the saved copies (allocated in ga_create, freed in ga_destroy); the caller owns
+ *     gradient buffers and every output buffer it passes in, and must keep a gradient buffer
+ *     unchanged until the work enqueued by the call that reads it has finished.
+ *   - Work is enqueued on the stream bound with ga_set_stream (default: the legacy default
+ *     stream) and the call returns after host bookkeeping; ga_get, ga_gap, ga_get_stats,
+ *     ga_export_state and the *_host calls synchronise that stream before returning.
+ *   - One engine serves one host thread at a time and lives on the device that was current
+ *     when it was created.
+ *   - No call aborts, traps or throws. Functions returning int give >= 0 on success or a
+ *     negative GA_ERR_* code; ga_last_error() then describes the failure. A CUDA error is
+ *     sticky: every later call on that engine returns GA_ERR_CUDA.
+ *   - Delays: k counts arrivals from 1; iter[i] (initially 0) is the number of arrivals applied
+ *     when worker i last pulled; the delay of an arrival is tau = k - iter[i] >= 1.
+ */
+#ifndef GA_H
+#define GA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ga_engine ga_engine;
+
+/* which master algorithm a push applies */
+enum {
+    GA_ASGD = 0, /* Algorithm "Momentum-ASGD: master" (Section 4)                      */
+    GA_SA = 1,   /* Algorithm "Staleness-Aware: master" (Section 4.1): step eta / tau   */
+    GA_GA = 2    /* Algorithm "Gap-Aware: master" (Section 5), parameter-wise Gap (5.3) */
+};
+
+enum { GA_OK = 0, GA_ERR_ARG = -1, GA_ERR_STATE = -2, GA_ERR_OOM = -3, GA_ERR_CUDA = -4 };
+
+/* vectors readable with ga_get */
+enum { GA_THETA = 0, GA_V = 1, GA_M = 2, GA_C = 3 };
+
+/* options for ga_set_option */
+enum {
+    GA_OPT_C_ORDER = 0, /* 0 (default): the Gap of arrival k uses C as it stands after arrival
+                           k-1, and m is then refreshed with the master's new v. 1: "Adam order":
+                           m is first refreshed with (gamma v + g)^2 of the raw gradient (the
+                           printed line of the C algorithm), then C, Gap and the step follow. */
+    GA_OPT_MATH = 1,    /* 0 (default): every operation IEEE round-to-nearest, in the order of
+                           the algorithms. 1: fast: approximate reciprocal and square root, one
+                           division per element (g*C/(|theta-theta^i|+C)); a few ulp off. */
+    GA_OPT_STATS = 2,   /* 1: every GA push also reduces sum and max of the Gap over all
+                           parameters (the quantity the paper logs per epoch, Appendix
+                           "Gap and Delay"); read with ga_get_stats. Default 0. */
+    GA_OPT_WINDOW = 3   /* 1..16 (default 16): most arrivals fused into one launch by
+                           ga_push_batch. */
+};
+
+#define GA_MAX_WINDOW 16
+
+/* Create a master for n_params parameters and n_workers workers. lr is eta (and eta_max of the
+ * C algorithm), momentum is gamma (|gamma| < 1; Section 3, no dampening), c_beta is beta_1 of
+ * Algorithm "C Coefficient Calculation" (0 <= c_beta < 1; the paper uses 0.999; eps is 1e-8).
+ * All state starts at 0: theta = v = m = 0, every saved copy = 0, no arrivals, iter[] = 0.
+ * Returns NULL on invalid arguments or allocation failure (see ga_last_error). */
+ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, float c_beta,
+                     int variant);
+
+/* Free everything the engine owns. NULL is accepted. Synchronises the bound stream first. */
+void ga_destroy(ga_engine* e);
+
+/* Enqueue all later work of this engine on cuda_stream (a cudaStream_t; NULL = default stream). */
+int ga_set_stream(ga_engine* e, void* cuda_stream);
+
+/* theta <- theta0 and every worker's saved copy <- theta0 ("Initialize theta^i = theta_0",
+ * Algorithm "DANA-Gap-Aware: master" line 1; the same convention is used for GA); v, m, the
+ * arrival counter and iter[] are reset to 0. theta0_dev: n_params floats on the device. */
+int ga_set_params(ga_engine* e, const float* theta0_dev);
+
+/* "Send theta to worker i" (Algorithm "Momentum-ASGD: worker": "Receive parameters"): copies the
+ * master parameters into worker's saved copy with TMA bulk copies, records iter[worker] <-
+ * arrivals applied so far, and returns the device address of that copy (library-owned, stable for
+ * the engine's life; contents change at that worker's next pull or batched push). NULL on error. */
+const float* ga_pull(ga_engine* e, int worker);
+
+/* Device address of worker's saved copy theta^worker (n_params floats) without copying anything:
+ * the parameters that worker was last sent, from which it computes its next gradient
+ * (Algorithm "Momentum-ASGD: worker"). Read-only for the caller. NULL on error. */
+const float* ga_saved(ga_engine* e, int worker);
+
+/* Apply one arriving gradient from `worker` (one iteration of the master algorithm of the
+ * engine's variant, without the final "send"): delay, [C, Gap, penalised gradient], momentum,
+ * step, [refresh of m]. grad_dev: n_params floats, unchanged until the work completes.
+ * Returns the delay tau >= 1 of this arrival, or a negative error. A worker may push again
+ * without pulling; its Gap is then still measured against its last saved copy. */
+int64_t ga_push(ga_engine* e, int worker, const float* grad_dev);
+
+/* K arrivals in FIFO order (Appendix "Algorithms": "the master's scheme is a simple FIFO"),
+ * each followed at once by that worker's pull -- the "Save and send current parameters" line of
+ * Algorithm "Gap-Aware: master". Equivalent to { ga_push(schedule[j], grads[j]);
+ * ga_pull(schedule[j]); } for j = 0..K-1, but up to GA_OPT_WINDOW consecutive arrivals are applied
+ * by one kernel that reads and writes theta, v, m once (legal because every step is independent
+ * per parameter, Section 5.3). A window is cut where a worker repeats. schedule_host: K worker
+ * ids; grads_host: K device pointers (a HOST array of device pointers); delays_out_host: K delays,
+ * may be NULL. K >= 0. Returns the number of kernel launches used, or a negative error (nothing
+ * is applied on an argument error). */
+int ga_push_batch(ga_engine* e, const int* schedule_host, const float* const* grads_host, int K,
+                  int64_t* delays_out_host);
+
+/* As ga_push_batch, for callers whose gradients and results live in HOST memory (pinned memory
+ * gives full PCIe speed): grads_host[j] points to n_params floats on the host; when
+ * sent_out_host is not NULL, sent_out_host[j] receives the parameters sent to worker
+ * schedule[j] after its arrival (n_params floats each). The parameter range is processed in
+ * chunks so that host-to-device copies, the update kernel and device-to-host copies overlap.
+ * Synchronous: returns when all results are in host memory. */
+int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* const* grads_host,
+                       int K, int64_t* delays_out_host, float* const* sent_out_host);
+
+/* Copy theta, v, m (which = GA_THETA, GA_V, GA_M) or the coefficient C derived from m as it
+ * stands (GA_C; last two lines of the C algorithm) into out_dev (n_params floats). */
+int ga_get(ga_engine* e, int which, float* out_dev);
+
+/* The parameter-wise Gap |theta - theta^worker| / C + 1 (Section 5.3) of `worker` against the
+ * master as it stands, into gap_out_dev (n_params floats). Changes no state. */
+int ga_gap(ga_engine* e, int worker, float* gap_out_dev);
+
+int ga_set_option(ga_engine* e, int key, double value);
+
+/* Sum and maximum over all parameters of the Gap used by the most recent GA arrival (needs
+ * GA_OPT_STATS = 1 before that push). GA_ERR_STATE when none is available. */
+int ga_get_stats(ga_engine* e, double* sum_gap, double* max_gap);
+
+/* Arrivals applied so far, and iter[worker]. Negative on error. */
+int64_t ga_num_arrivals(ga_engine* e);
+int64_t ga_worker_iter(ga_engine* e, int worker);
+
+/* Checkpoint: all state needed to continue bit-identically (hyper-parameters, options, counters,
+ * iter[], theta, v, m, saved copies). ga_export_state returns the number of bytes needed; it
+ * writes them when cap is large enough (buf_host may be NULL to query). ga_import_state needs an
+ * engine created with the same n_params and n_workers. */
+size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap);
+int ga_import_state(ga_engine* e, const void* buf_host, size_t len);
+
+/* Message for the calling thread's most recent failure ("" if none). Never NULL. */
+const char* ga_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GA_H */

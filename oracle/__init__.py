@@ -42,6 +42,9 @@ def _bind(path):
     lib.gao_k_done.argtypes = [c.c_void_p]
     lib.gao_iter.restype = c.c_int64
     lib.gao_iter.argtypes = [c.c_void_p, c.c_int]
+    lib.gao_set_state.argtypes = [c.c_void_p] * 6 + [c.c_int64, c.c_int64]
+    lib.gao_k_c.restype = c.c_int64
+    lib.gao_k_c.argtypes = [c.c_void_p]
     lib.gao_stats.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
     lib.gao_get.restype = c.c_int
     lib.gao_get.argtypes = [c.c_void_p, c.c_int, c.c_void_p]
@@ -132,6 +135,19 @@ class Oracle:
         s, m = ctypes.c_double(), ctypes.c_double()
         self._l.gao_stats(self._h, ctypes.byref(s), ctypes.byref(m))
         return s.value, m.value
+
+    def state(self):
+        """(theta, v, m, saved[N][d], iter[N], k_done, k_c); vectors as float64."""
+        saved = np.stack([self.saved(i) for i in range(self.n)])
+        iters = np.asarray([self.iter(i) for i in range(self.n)], dtype=np.int64)
+        return (self.get(self.THETA), self.get(self.V), self.get(self.M), saved, iters,
+                self.k_done, int(self._l.gao_k_c(self._h)))
+
+    def set_state(self, theta, v, m, saved, iters, k_done, k_c):
+        a = [np.ascontiguousarray(x, dtype=np.float64) for x in (theta, v, m, saved)]
+        assert a[0].shape == (self.d,) and a[3].shape == (self.n, self.d)
+        it = np.ascontiguousarray(iters, dtype=np.int64)
+        self._l.gao_set_state(self._h, *(x.ctypes.data for x in a), it.ctypes.data, k_done, k_c)
 
     @property
     def k_done(self):

@@ -150,6 +150,16 @@ struct Master {
         return tau;
     }
 
+    // Overwrite the whole state (used by tests that start both precisions from one state).
+    void set_state(const double* th, const double* vv, const double* mm, const double* sv,
+                   const int64_t* it, int64_t kd, int64_t kc) {
+        for (int64_t j = 0; j < d; ++j) { theta[j] = (T)th[j]; v[j] = (T)vv[j]; m[j] = (T)mm[j]; }
+        for (size_t q = 0; q < (size_t)n_workers * d; ++q) saved[q] = (T)sv[q];
+        for (int i = 0; i < n_workers; ++i) iter[i] = it[i];
+        k_done = kd;
+        k_c = kc;
+    }
+
     // Gap of worker i against the master as it stands; changes nothing.
     void gap(int i, double* out) const {
         const T* s = &saved[(size_t)i * d];
@@ -233,6 +243,13 @@ int64_t gao_push(void* p, int worker, const float* grad) { auto* h = (Handle*)p;
 void gao_gap(void* p, int worker, double* out) { auto* h = (Handle*)p; DISPATCH(h, gap(worker, out)); }
 int64_t gao_k_done(void* p) { auto* h = (Handle*)p; return h->precision == 32 ? h->f->k_done : h->g->k_done; }
 int64_t gao_iter(void* p, int worker) { auto* h = (Handle*)p; return h->precision == 32 ? h->f->iter[worker] : h->g->iter[worker]; }
+
+void gao_set_state(void* p, const double* th, const double* v, const double* m, const double* saved,
+                   const int64_t* iter, int64_t k_done, int64_t k_c) {
+    auto* h = (Handle*)p;
+    DISPATCH(h, set_state(th, v, m, saved, iter, k_done, k_c));
+}
+int64_t gao_k_c(void* p) { auto* h = (Handle*)p; return h->precision == 32 ? h->f->k_c : h->g->k_c; }
 
 void gao_stats(void* p, double* sum_gap, double* max_gap) {
     auto* h = (Handle*)p;

@@ -1,0 +1,600 @@
+// Host side of the C ABI declared in include/ga.h: argument checks, the master's integer
+// bookkeeping (arrival counter, iter[], delays, bias-correction scalars, window cutting) and
+// kernel launches. All arithmetic on parameters happens in the kernels of ga_kernels.cuh.
+#include "ga.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "ga_kernels.cuh"
+
+namespace {
+
+thread_local std::string g_error;
+
+int fail(int code, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_error = buf;
+    return code;
+}
+
+constexpr long long kRowAlign = 32;            // floats: rows start on 128-byte boundaries
+constexpr long long kHostChunk = 4ll << 20;    // floats per chunk of the host-buffer path
+constexpr uint32_t kStateMagic = 0x47415331;   // "GAS1"
+
+}  // namespace
+
+struct ga_engine {
+    long long d = 0, stride = 0;  // parameters; padded row length in floats
+    int n_workers = 0, variant = GA_GA, device = 0;
+    float lr = 0, gamma = 0, beta = 0, eps = 1e-8f;
+    int c_order = 0, fast_math = 0, stats = 0, window = GA_MAX_WINDOW;
+    float *theta = nullptr, *vel = nullptr, *mom = nullptr, *saved = nullptr;
+    std::vector<int64_t> iter;
+    int64_t k_done = 0, k_c = 0;
+    cudaStream_t stream = nullptr;
+    bool cuda_failed = false;
+    // statistics
+    ga::StatsPartial* partials = nullptr;
+    double* stats_dev = nullptr;   // kMaxWindow x {sum, max}
+    int stats_blocks = 0;
+    bool stats_valid = false;
+    int stats_slot = 0;
+    // pull kernel error flag
+    int* pull_err = nullptr;
+    // host-buffer path
+    float* stage[2] = {nullptr, nullptr};
+    long long stage_elems = 0;
+    cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+    cudaEvent_t ev_h2d[2] = {nullptr, nullptr}, ev_kernel[2] = {nullptr, nullptr}, ev_prev = nullptr;
+
+    float* row(int i) const { return saved + (size_t)i * stride; }
+    ga::Hyper hyper() const {
+        ga::Hyper h;
+        h.eta_max = lr;
+        h.gamma = gamma;
+        h.beta = beta;
+        h.one_minus_beta = (float)(1.0 - (double)beta);
+        h.eps = eps;
+        return h;
+    }
+    // 1/(1-beta^k) for the C in force after k refreshes of m; 0 before the first (C = eta_max*eps)
+    float inv_bias(int64_t k) const {
+        if (k <= 0) return 0.f;
+        return (float)(1.0 / (1.0 - std::pow((double)beta, (double)k)));
+    }
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+int cuda_fail(ga_engine* e, cudaError_t err, const char* what) {
+    if (e) e->cuda_failed = true;
+    return fail(GA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(err));
+}
+
+#define GA_CUDA(e, call)                                             \
+    do {                                                             \
+        cudaError_t err__ = (call);                                  \
+        if (err__ != cudaSuccess) return cuda_fail((e), err__, #call); \
+    } while (0)
+
+int check_engine(ga_engine* e) {
+    if (!e) return fail(GA_ERR_ARG, "engine is NULL");
+    if (e->cuda_failed) return fail(GA_ERR_CUDA, "engine is unusable after an earlier CUDA error");
+    return GA_OK;
+}
+
+int check_worker(ga_engine* e, int worker) {
+    if (worker < 0 || worker >= e->n_workers)
+        return fail(GA_ERR_ARG, "worker %d out of range [0, %d)", worker, e->n_workers);
+    return GA_OK;
+}
+
+int check_dev_ptr(const void* p, const char* name) {
+    if (!p) return fail(GA_ERR_ARG, "%s is NULL", name);
+    if ((uintptr_t)p % 16) return fail(GA_ERR_ARG, "%s is not 16-byte aligned", name);
+    return GA_OK;
+}
+
+// After a synchronisation: did a bulk-copy wait of a pull kernel run out?
+int check_pull_flag(ga_engine* e) {
+    int flag = 0;
+    GA_CUDA(e, cudaMemcpy(&flag, e->pull_err, sizeof flag, cudaMemcpyDeviceToHost));
+    if (flag) {
+        e->cuda_failed = true;
+        return fail(GA_ERR_CUDA, "a bulk copy of ga_pull did not complete within its wait limit");
+    }
+    return GA_OK;
+}
+
+int grid_1d(long long n, int threads, int cap) {
+    long long g = (n + threads - 1) / threads;
+    if (g < 1) g = 1;
+    return (int)(g < cap ? g : cap);
+}
+
+// ----------------------------------------------------------------------------- launch
+template <int VARIANT, bool EXACT, int C_ORDER, bool STATS>
+void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st) {
+    constexpr int B = 4;
+    const long long nvec = vec_end - vec_begin;
+    long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
+    if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
+    ga::ga_window_kernel<VARIANT, EXACT, C_ORDER, STATS, B><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
+        e->theta, e->vel, e->mom, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
+    if (STATS) {
+        ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev);
+    }
+}
+
+int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st,
+                  bool allow_stats = true) {
+    if (vec_end <= vec_begin || w.K <= 0) return GA_OK;
+    const bool exact = !e->fast_math;
+    const bool stats = allow_stats && e->stats && e->variant == GA_GA;
+    if (e->variant == GA_ASGD) launch_window_t<ga::ASGD, true, 0, false>(e, w, vec_begin, vec_end, st);
+    else if (e->variant == GA_SA) launch_window_t<ga::SA, true, 0, false>(e, w, vec_begin, vec_end, st);
+    else {
+#define GA_CASE(EX, CO, ST) launch_window_t<ga::GA, EX, CO, ST>(e, w, vec_begin, vec_end, st)
+        if (exact) {
+            if (e->c_order == 0) { if (stats) GA_CASE(true, 0, true); else GA_CASE(true, 0, false); }
+            else { if (stats) GA_CASE(true, 1, true); else GA_CASE(true, 1, false); }
+        } else {
+            if (e->c_order == 0) { if (stats) GA_CASE(false, 0, true); else GA_CASE(false, 0, false); }
+            else { if (stats) GA_CASE(false, 1, true); else GA_CASE(false, 1, false); }
+        }
+#undef GA_CASE
+    }
+    GA_CUDA(e, cudaGetLastError());
+    if (stats) { e->stats_valid = true; e->stats_slot = w.K - 1; }
+    return GA_OK;
+}
+
+// Fill the arrival table for arrivals j0..j0+K-1 of a batch and advance the counters.
+void fill_window(ga_engine* e, ga::Window& w, const int* workers, const float* const* grads, int K,
+                 bool with_pull, int64_t* delays) {
+    w.K = K;
+    w.write_saved = with_pull ? 1 : 0;
+    w.grad_offset = 0;
+    for (int j = 0; j < K; ++j) {
+        const int i = workers[j];
+        const int64_t k = e->k_done + 1;
+        const int64_t tau = k - e->iter[i];
+        if (delays) delays[j] = tau;
+        w.grad[j] = grads[j];
+        w.saved[j] = e->row(i);
+        w.eta_eff[j] = e->variant == GA_SA ? e->lr / (float)tau : e->lr;
+        if (e->variant == GA_GA) {
+            // the C in force for this arrival: after k_c refreshes (lagged order), or after
+            // this arrival's own refresh (Adam order)
+            w.inv_bias[j] = e->inv_bias(e->c_order == 0 ? e->k_c : e->k_c + 1);
+            e->k_c += 1;
+        } else {
+            w.inv_bias[j] = 0.f;
+        }
+        e->k_done = k;
+        if (with_pull) e->iter[i] = k;
+    }
+    for (int j = K; j < ga::kMaxWindow; ++j) {
+        w.grad[j] = nullptr;
+        w.saved[j] = nullptr;
+        w.inv_bias[j] = 0.f;
+        w.eta_eff[j] = 0.f;
+    }
+}
+
+// Length of the next window starting at schedule[pos]: at most `window` arrivals, cut where a
+// worker would appear a second time.
+int next_window(const int* schedule, int pos, int K, int window) {
+    int n = 0;
+    while (pos + n < K && n < window) {
+        bool repeat = false;
+        for (int q = 0; q < n; ++q) repeat |= schedule[pos + q] == schedule[pos + n];
+        if (repeat) break;
+        ++n;
+    }
+    return n;
+}
+
+int validate_batch(ga_engine* e, const int* schedule, const void* const* bufs, int K, bool device_ptrs) {
+    if (K < 0) return fail(GA_ERR_ARG, "K = %d is negative", K);
+    if (K > 0 && (!schedule || !bufs)) return fail(GA_ERR_ARG, "schedule or gradient array is NULL");
+    for (int j = 0; j < K; ++j) {
+        if (int rc = check_worker(e, schedule[j])) return rc;
+        if (!bufs[j]) return fail(GA_ERR_ARG, "gradient %d is NULL", j);
+        if (device_ptrs && (uintptr_t)bufs[j] % 16) return fail(GA_ERR_ARG, "gradient %d is not 16-byte aligned", j);
+    }
+    return GA_OK;
+}
+
+int ensure_host_path(ga_engine* e) {
+    if (e->stage[0]) return GA_OK;
+    const long long chunk = e->stride < kHostChunk ? e->stride : kHostChunk;
+    e->stage_elems = chunk;
+    for (int s = 0; s < 2; ++s) {
+        if (cudaMalloc(&e->stage[s], sizeof(float) * (size_t)chunk * ga::kMaxWindow) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(GA_ERR_OOM, "cannot allocate staging buffers for the host-buffer path");
+        }
+        GA_CUDA(e, cudaEventCreateWithFlags(&e->ev_h2d[s], cudaEventDisableTiming));
+        GA_CUDA(e, cudaEventCreateWithFlags(&e->ev_kernel[s], cudaEventDisableTiming));
+    }
+    GA_CUDA(e, cudaEventCreateWithFlags(&e->ev_prev, cudaEventDisableTiming));
+    GA_CUDA(e, cudaStreamCreateWithFlags(&e->s_h2d, cudaStreamNonBlocking));
+    GA_CUDA(e, cudaStreamCreateWithFlags(&e->s_d2h, cudaStreamNonBlocking));
+    return GA_OK;
+}
+
+}  // namespace
+
+// ================================================================================= C ABI
+extern "C" {
+
+const char* ga_last_error(void) { return g_error.c_str(); }
+
+ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, float c_beta, int variant) {
+    g_error.clear();
+    if (n_params == 0 || n_params > (size_t)1 << 40) { fail(GA_ERR_ARG, "n_params out of range"); return nullptr; }
+    if (n_workers <= 0 || n_workers > 65536) { fail(GA_ERR_ARG, "n_workers out of range"); return nullptr; }
+    if (!(lr > 0.f) || !std::isfinite(lr)) { fail(GA_ERR_ARG, "lr must be positive and finite"); return nullptr; }
+    if (!(std::fabs(momentum) < 1.f)) { fail(GA_ERR_ARG, "|momentum| must be < 1"); return nullptr; }
+    if (!(c_beta >= 0.f && c_beta < 1.f)) { fail(GA_ERR_ARG, "c_beta must be in [0, 1)"); return nullptr; }
+    if (variant != GA_ASGD && variant != GA_SA && variant != GA_GA) { fail(GA_ERR_ARG, "unknown variant %d", variant); return nullptr; }
+    ga_engine* e = new (std::nothrow) ga_engine();
+    if (!e) { fail(GA_ERR_OOM, "out of host memory"); return nullptr; }
+    e->d = (long long)n_params;
+    e->stride = (e->d + kRowAlign - 1) / kRowAlign * kRowAlign;
+    e->n_workers = n_workers;
+    e->lr = lr;
+    e->gamma = momentum;
+    e->beta = c_beta;
+    e->variant = variant;
+    e->iter.assign(n_workers, 0);
+    if (cudaGetDevice(&e->device) != cudaSuccess) {
+        fail(GA_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+        delete e;
+        return nullptr;
+    }
+    cudaDeviceProp prop;
+    int sms = 148;
+    if (cudaGetDeviceProperties(&prop, e->device) == cudaSuccess) sms = prop.multiProcessorCount;
+    e->stats_blocks = sms * 8;
+    const size_t row_bytes = sizeof(float) * (size_t)e->stride;
+    bool ok = cudaMalloc(&e->theta, row_bytes) == cudaSuccess && cudaMalloc(&e->vel, row_bytes) == cudaSuccess &&
+              cudaMalloc(&e->mom, row_bytes) == cudaSuccess &&
+              cudaMalloc(&e->saved, row_bytes * (size_t)n_workers) == cudaSuccess &&
+              cudaMalloc(&e->partials, sizeof(ga::StatsPartial) * (size_t)e->stats_blocks * ga::kMaxWindow) == cudaSuccess &&
+              cudaMalloc(&e->stats_dev, sizeof(double) * 2 * ga::kMaxWindow) == cudaSuccess &&
+              cudaMalloc(&e->pull_err, sizeof(int)) == cudaSuccess;
+    if (ok) {
+        ok = cudaMemset(e->theta, 0, row_bytes) == cudaSuccess && cudaMemset(e->vel, 0, row_bytes) == cudaSuccess &&
+             cudaMemset(e->mom, 0, row_bytes) == cudaSuccess &&
+             cudaMemset(e->saved, 0, row_bytes * (size_t)n_workers) == cudaSuccess &&
+             cudaMemset(e->pull_err, 0, sizeof(int)) == cudaSuccess &&
+             cudaFuncSetAttribute(ga::ga_pull_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  ga::kPullStages * ga::kPullChunk) == cudaSuccess &&
+             cudaDeviceSynchronize() == cudaSuccess;
+    }
+    if (!ok) {
+        cudaError_t err = cudaGetLastError();
+        fail(err == cudaErrorMemoryAllocation ? GA_ERR_OOM : GA_ERR_CUDA, "ga_create: %s", cudaGetErrorString(err));
+        ga_destroy(e);
+        return nullptr;
+    }
+    return e;
+}
+
+void ga_destroy(ga_engine* e) {
+    if (!e) return;
+    DeviceGuard guard(e->device);
+    cudaStreamSynchronize(e->stream);
+    cudaFree(e->theta);
+    cudaFree(e->vel);
+    cudaFree(e->mom);
+    cudaFree(e->saved);
+    cudaFree(e->partials);
+    cudaFree(e->stats_dev);
+    cudaFree(e->pull_err);
+    for (int s = 0; s < 2; ++s) {
+        cudaFree(e->stage[s]);
+        if (e->ev_h2d[s]) cudaEventDestroy(e->ev_h2d[s]);
+        if (e->ev_kernel[s]) cudaEventDestroy(e->ev_kernel[s]);
+    }
+    if (e->ev_prev) cudaEventDestroy(e->ev_prev);
+    if (e->s_h2d) cudaStreamDestroy(e->s_h2d);
+    if (e->s_d2h) cudaStreamDestroy(e->s_d2h);
+    cudaGetLastError();
+    delete e;
+}
+
+int ga_set_stream(ga_engine* e, void* cuda_stream) {
+    if (int rc = check_engine(e)) return rc;
+    e->stream = (cudaStream_t)cuda_stream;
+    return GA_OK;
+}
+
+int ga_set_params(ga_engine* e, const float* theta0_dev) {
+    if (int rc = check_engine(e)) return rc;
+    if (int rc = check_dev_ptr(theta0_dev, "theta0_dev")) return rc;
+    DeviceGuard guard(e->device);
+    ga::ga_set_params_kernel<<<grid_1d(e->stride, 256, 148 * 8), 256, 0, e->stream>>>(
+        theta0_dev, e->theta, e->vel, e->mom, e->saved, e->n_workers, e->d, e->stride);
+    GA_CUDA(e, cudaGetLastError());
+    std::fill(e->iter.begin(), e->iter.end(), 0);
+    e->k_done = 0;
+    e->k_c = 0;
+    e->stats_valid = false;
+    return GA_OK;
+}
+
+const float* ga_pull(ga_engine* e, int worker) {
+    if (check_engine(e) || check_worker(e, worker)) return nullptr;
+    DeviceGuard guard(e->device);
+    const long long bytes = e->stride * (long long)sizeof(float);
+    const long long chunks = (bytes + ga::kPullChunk - 1) / ga::kPullChunk;
+    const int grid = (int)(chunks < 148 * 3 ? chunks : 148 * 3);
+    ga::ga_pull_bulk_kernel<<<grid, 32, ga::kPullStages * ga::kPullChunk, e->stream>>>(
+        e->theta, e->row(worker), bytes, e->pull_err);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { cuda_fail(e, err, "ga_pull launch"); return nullptr; }
+    e->iter[worker] = e->k_done;
+    return e->row(worker);
+}
+
+const float* ga_saved(ga_engine* e, int worker) {
+    if (check_engine(e) || check_worker(e, worker)) return nullptr;
+    return e->row(worker);
+}
+
+int64_t ga_push(ga_engine* e, int worker, const float* grad_dev) {
+    if (int rc = check_engine(e)) return rc;
+    if (int rc = check_worker(e, worker)) return rc;
+    if (int rc = check_dev_ptr(grad_dev, "grad_dev")) return rc;
+    DeviceGuard guard(e->device);
+    ga::Window w;
+    int64_t tau = 0;
+    fill_window(e, w, &worker, &grad_dev, 1, /*with_pull=*/false, &tau);
+    if (int rc = launch_window(e, w, 0, e->stride / 4, e->stream)) return rc;
+    return tau;
+}
+
+int ga_push_batch(ga_engine* e, const int* schedule_host, const float* const* grads_host, int K,
+                  int64_t* delays_out_host) {
+    if (int rc = check_engine(e)) return rc;
+    if (int rc = validate_batch(e, schedule_host, (const void* const*)grads_host, K, true)) return rc;
+    DeviceGuard guard(e->device);
+    int launches = 0;
+    for (int pos = 0; pos < K;) {
+        const int n = next_window(schedule_host, pos, K, e->window);
+        ga::Window w;
+        fill_window(e, w, schedule_host + pos, grads_host + pos, n, true,
+                    delays_out_host ? delays_out_host + pos : nullptr);
+        if (int rc = launch_window(e, w, 0, e->stride / 4, e->stream)) return rc;
+        ++launches;
+        pos += n;
+    }
+    return launches;
+}
+
+int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* const* grads_host, int K,
+                       int64_t* delays_out_host, float* const* sent_out_host) {
+    if (int rc = check_engine(e)) return rc;
+    if (int rc = validate_batch(e, schedule_host, (const void* const*)grads_host, K, false)) return rc;
+    if (sent_out_host)
+        for (int j = 0; j < K; ++j)
+            if (!sent_out_host[j]) return fail(GA_ERR_ARG, "sent_out_host[%d] is NULL", j);
+    DeviceGuard guard(e->device);
+    if (int rc = ensure_host_path(e)) return rc;
+    int launches = 0;
+    const long long chunk = e->stage_elems;
+    // the copy streams start after everything already enqueued on the engine's stream
+    GA_CUDA(e, cudaEventRecord(e->ev_prev, e->stream));
+    GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_prev, 0));
+    GA_CUDA(e, cudaStreamWaitEvent(e->s_d2h, e->ev_prev, 0));
+    for (int pos = 0; pos < K;) {
+        const int n = next_window(schedule_host, pos, K, e->window);
+        ga::Window w;
+        const float* staged[ga::kMaxWindow] = {};
+        fill_window(e, w, schedule_host + pos, staged, n, true, delays_out_host ? delays_out_host + pos : nullptr);
+        long long c_index = 0;
+        for (long long c0 = 0; c0 < e->stride; c0 += chunk, ++c_index) {
+            const int s = (int)(c_index & 1);
+            const long long c1 = c0 + chunk < e->stride ? c0 + chunk : e->stride;
+            const long long valid = (c1 < e->d ? c1 : e->d) - c0;   // floats the caller's buffers hold
+            // staging buffer s is free once the kernel of chunk c_index-2 has run
+            if (c_index >= 2) GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_kernel[s], 0));
+            for (int j = 0; j < n; ++j) {
+                float* dst = e->stage[s] + (size_t)j * chunk;
+                if (valid > 0)
+                    GA_CUDA(e, cudaMemcpyAsync(dst, grads_host[pos + j] + c0, sizeof(float) * (size_t)valid,
+                                               cudaMemcpyHostToDevice, e->s_h2d));
+                w.grad[j] = dst;
+            }
+            GA_CUDA(e, cudaEventRecord(e->ev_h2d[s], e->s_h2d));
+            GA_CUDA(e, cudaStreamWaitEvent(e->stream, e->ev_h2d[s], 0));
+            w.grad_offset = c0;
+            if (int rc = launch_window(e, w, c0 / 4, c1 / 4, e->stream, /*allow_stats=*/false)) return rc;
+            ++launches;
+            GA_CUDA(e, cudaEventRecord(e->ev_kernel[s], e->stream));
+            if (sent_out_host && valid > 0) {
+                GA_CUDA(e, cudaStreamWaitEvent(e->s_d2h, e->ev_kernel[s], 0));
+                for (int j = 0; j < n; ++j)
+                    GA_CUDA(e, cudaMemcpyAsync(sent_out_host[pos + j] + c0, e->row(schedule_host[pos + j]) + c0,
+                                               sizeof(float) * (size_t)valid, cudaMemcpyDeviceToHost, e->s_d2h));
+            }
+        }
+        // a later window may rewrite the rows being read back and reuse the staging buffers
+        GA_CUDA(e, cudaStreamSynchronize(e->s_h2d));
+        GA_CUDA(e, cudaStreamSynchronize(e->stream));
+        GA_CUDA(e, cudaStreamSynchronize(e->s_d2h));
+        pos += n;
+    }
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    return launches;
+}
+
+int ga_get(ga_engine* e, int which, float* out_dev) {
+    if (int rc = check_engine(e)) return rc;
+    if (int rc = check_dev_ptr(out_dev, "out_dev")) return rc;
+    DeviceGuard guard(e->device);
+    const float* src = which == GA_THETA ? e->theta : which == GA_V ? e->vel : which == GA_M ? e->mom : nullptr;
+    if (src) {
+        GA_CUDA(e, cudaMemcpyAsync(out_dev, src, sizeof(float) * (size_t)e->d, cudaMemcpyDeviceToDevice, e->stream));
+    } else if (which == GA_C) {
+        ga::ga_coeff_kernel<<<grid_1d(e->d, 256, 148 * 8), 256, 0, e->stream>>>(e->mom, e->inv_bias(e->k_c),
+                                                                               e->hyper(), e->d, out_dev);
+        GA_CUDA(e, cudaGetLastError());
+    } else {
+        return fail(GA_ERR_ARG, "unknown vector %d", which);
+    }
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    return check_pull_flag(e);
+}
+
+int ga_gap(ga_engine* e, int worker, float* gap_out_dev) {
+    if (int rc = check_engine(e)) return rc;
+    if (int rc = check_worker(e, worker)) return rc;
+    if (int rc = check_dev_ptr(gap_out_dev, "gap_out_dev")) return rc;
+    DeviceGuard guard(e->device);
+    ga::ga_gap_kernel<<<grid_1d(e->d, 256, 148 * 8), 256, 0, e->stream>>>(
+        e->theta, e->row(worker), e->mom, e->inv_bias(e->k_c), e->hyper(), e->d, gap_out_dev);
+    GA_CUDA(e, cudaGetLastError());
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    return GA_OK;
+}
+
+int ga_set_option(ga_engine* e, int key, double value) {
+    if (int rc = check_engine(e)) return rc;
+    const int v = (int)value;
+    switch (key) {
+        case GA_OPT_C_ORDER:
+            if (v != 0 && v != 1) return fail(GA_ERR_ARG, "GA_OPT_C_ORDER must be 0 or 1");
+            if (e->k_done != 0) return fail(GA_ERR_STATE, "GA_OPT_C_ORDER can only change before the first arrival");
+            e->c_order = v;
+            return GA_OK;
+        case GA_OPT_MATH:
+            if (v != 0 && v != 1) return fail(GA_ERR_ARG, "GA_OPT_MATH must be 0 or 1");
+            e->fast_math = v;
+            return GA_OK;
+        case GA_OPT_STATS:
+            if (v != 0 && v != 1) return fail(GA_ERR_ARG, "GA_OPT_STATS must be 0 or 1");
+            e->stats = v;
+            if (!v) e->stats_valid = false;
+            return GA_OK;
+        case GA_OPT_WINDOW:
+            if (v < 1 || v > GA_MAX_WINDOW) return fail(GA_ERR_ARG, "GA_OPT_WINDOW must be in [1, %d]", GA_MAX_WINDOW);
+            e->window = v;
+            return GA_OK;
+        default:
+            return fail(GA_ERR_ARG, "unknown option %d", key);
+    }
+}
+
+int ga_get_stats(ga_engine* e, double* sum_gap, double* max_gap) {
+    if (int rc = check_engine(e)) return rc;
+    if (!sum_gap || !max_gap) return fail(GA_ERR_ARG, "output pointer is NULL");
+    if (!e->stats_valid) return fail(GA_ERR_STATE, "no Gap statistics: enable GA_OPT_STATS before a GA push");
+    DeviceGuard guard(e->device);
+    double host[2 * ga::kMaxWindow];
+    GA_CUDA(e, cudaMemcpyAsync(host, e->stats_dev, sizeof host, cudaMemcpyDeviceToHost, e->stream));
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    *sum_gap = host[2 * e->stats_slot];
+    *max_gap = host[2 * e->stats_slot + 1];
+    return GA_OK;
+}
+
+int64_t ga_num_arrivals(ga_engine* e) {
+    if (int rc = check_engine(e)) return rc;
+    return e->k_done;
+}
+
+int64_t ga_worker_iter(ga_engine* e, int worker) {
+    if (int rc = check_engine(e)) return rc;
+    if (int rc = check_worker(e, worker)) return rc;
+    return e->iter[worker];
+}
+
+// ---- checkpoint layout: header, iter[n_workers], theta[d], v[d], m[d], saved[n_workers][d]
+struct StateHeader {
+    uint32_t magic, version;
+    int64_t d, n_workers, k_done, k_c;
+    float lr, gamma, beta, eps;
+    int32_t variant, c_order, fast_math, stats, window, reserved;
+};
+
+size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
+    if (check_engine(e)) return 0;
+    const size_t vec = sizeof(float) * (size_t)e->d;
+    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * (3 + (size_t)e->n_workers);
+    if (!buf_host || cap < need) return need;
+    DeviceGuard guard(e->device);
+    StateHeader h{};
+    h.magic = kStateMagic; h.version = 1;
+    h.d = e->d; h.n_workers = e->n_workers; h.k_done = e->k_done; h.k_c = e->k_c;
+    h.lr = e->lr; h.gamma = e->gamma; h.beta = e->beta; h.eps = e->eps;
+    h.variant = e->variant; h.c_order = e->c_order; h.fast_math = e->fast_math; h.stats = e->stats; h.window = e->window;
+    char* p = (char*)buf_host;
+    std::memcpy(p, &h, sizeof h); p += sizeof h;
+    std::memcpy(p, e->iter.data(), sizeof(int64_t) * e->n_workers); p += sizeof(int64_t) * e->n_workers;
+    const float* vecs[3] = {e->theta, e->vel, e->mom};
+    cudaError_t err = cudaSuccess;
+    for (int q = 0; q < 3 && err == cudaSuccess; ++q, p += vec)
+        err = cudaMemcpyAsync(p, vecs[q], vec, cudaMemcpyDeviceToHost, e->stream);
+    for (int i = 0; i < e->n_workers && err == cudaSuccess; ++i, p += vec)
+        err = cudaMemcpyAsync(p, e->row(i), vec, cudaMemcpyDeviceToHost, e->stream);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(e->stream);
+    if (err != cudaSuccess) { cuda_fail(e, err, "ga_export_state"); return 0; }
+    return need;
+}
+
+int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
+    if (int rc = check_engine(e)) return rc;
+    if (!buf_host || len < sizeof(StateHeader)) return fail(GA_ERR_ARG, "state buffer too short");
+    StateHeader h;
+    std::memcpy(&h, buf_host, sizeof h);
+    if (h.magic != kStateMagic || h.version != 1) return fail(GA_ERR_ARG, "not a state written by ga_export_state");
+    if (h.d != e->d || h.n_workers != e->n_workers)
+        return fail(GA_ERR_ARG, "state is for %lld parameters / %lld workers", (long long)h.d, (long long)h.n_workers);
+    const size_t vec = sizeof(float) * (size_t)e->d;
+    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * (3 + (size_t)e->n_workers);
+    if (len < need) return fail(GA_ERR_ARG, "state buffer truncated");
+    if (h.variant < GA_ASGD || h.variant > GA_GA || h.window < 1 || h.window > GA_MAX_WINDOW || h.k_done < 0 || h.k_c < 0)
+        return fail(GA_ERR_ARG, "state header holds invalid values");
+    DeviceGuard guard(e->device);
+    const char* p = (const char*)buf_host + sizeof h;
+    std::vector<int64_t> iter(e->n_workers);
+    std::memcpy(iter.data(), p, sizeof(int64_t) * e->n_workers); p += sizeof(int64_t) * e->n_workers;
+    float* vecs[3] = {e->theta, e->vel, e->mom};
+    for (int q = 0; q < 3; ++q, p += vec)
+        GA_CUDA(e, cudaMemcpyAsync(vecs[q], p, vec, cudaMemcpyHostToDevice, e->stream));
+    for (int i = 0; i < e->n_workers; ++i, p += vec)
+        GA_CUDA(e, cudaMemcpyAsync(e->row(i), p, vec, cudaMemcpyHostToDevice, e->stream));
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    e->iter = iter;
+    e->k_done = h.k_done; e->k_c = h.k_c;
+    e->lr = h.lr; e->gamma = h.gamma; e->beta = h.beta; e->eps = h.eps;
+    e->variant = h.variant; e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window;
+    e->stats_valid = false;
+    return GA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,401 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle.
+
+The fp32 oracle rounds exactly as the kernels' exact mode does, so whole trajectories are
+compared element by element and must agree within 1e-5*(1+|ref|) -- and, as measured, bit for
+bit. (The synthetic quadratic is unstable under the simulated delays for several of the
+configurations, so a trajectory-level tolerance would be meaningless for anything but an
+implementation that rounds identically; single arrivals from identical states are also
+compared with the fp64 oracle, and fast-math mode is held to the tolerance the same way.)
+"""
+import numpy as np
+import pytest
+
+import oracle
+import workloads as W
+from tests.oracle_run import run_oracle, within, worst
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5     # max |gpu - ref| <= TOL * (1 + |ref|)
+
+
+@pytest.fixture(scope="module")
+def P():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_1909_10802_b200 as pkg
+    pkg.lib()
+    W.cuda_lib()
+    return pkg
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+def _same(a, b):
+    """Equal element by element; NaN equals NaN (payload bits differ between CPU and GPU)."""
+    return np.array_equal(np.asarray(a, dtype=np.float32), np.asarray(b, dtype=np.float32), equal_nan=True)
+
+
+def _close(got, ref):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    fin = np.isfinite(ref)
+    if not np.array_equal(np.isnan(got), np.isnan(ref)):
+        return False
+    if not np.array_equal(got[~fin & ~np.isnan(ref)], ref[~fin & ~np.isnan(ref)]):
+        return False
+    return within(got[fin], ref[fin], TOL)
+
+
+def _compare_engine(P, run, o, idx=None, label=""):
+    """theta, v, m and derived C of the engine against the oracle (at idx if given)."""
+    import torch
+    sel = None if idx is None else torch.as_tensor(idx, device="cuda")
+    names = (("theta", P.GA_THETA, o.THETA), ("v", P.GA_V, o.V))
+    if run.engine.variant == P.GA_GA:
+        names += (("m", P.GA_M, o.M), ("C", P.GA_C, o.C))
+    for name, which, owhich in names:
+        got = run.engine.get(which)
+        got = _np(got if sel is None else got[sel])
+        ref = o.get(owhich)
+        assert _close(got, ref), f"{label}{name}: outside {TOL}*(1+|ref|)"
+        nbad = int(np.sum(~((got == ref.astype(np.float32)) | (np.isnan(got) & np.isnan(ref)))))
+        assert nbad == 0, f"{label}{name}: {nbad} elements differ from the fp32 oracle in some bit"
+
+
+# ----------------------------------------------------------------------------- generators
+@pytest.mark.parametrize("name", ["mini", "C1"])
+def test_device_generator_matches_cpu(P, name):
+    import torch
+    wl = W.config(name)
+    dev = wl.device()
+    t0 = torch.empty(wl.d, dtype=torch.float32, device="cuda")
+    dev.theta0(t0)
+    assert np.array_equal(_np(t0), wl.theta0())
+    g = torch.empty_like(t0)
+    for k in (1, 7):
+        dev.grad_ptr(k, t0.data_ptr(), g.data_ptr())
+        assert np.array_equal(_np(g), wl.grad(k, wl.theta0()))
+
+
+def test_device_generator_sparse_rows_and_subrange(P):
+    import torch
+    wl = W.Workload(name="emb", segments=[64 * 300, 5000], n_workers=2, arrivals=4, schedule_kind="ticks",
+                    seed=11, quad=False, emb_rows=300, emb_row=64, row_active_frac=0.1)
+    dev = wl.device()
+    z = torch.zeros(wl.d, dtype=torch.float32, device="cuda")
+    g = torch.empty_like(z)
+    dev.grad_ptr(3, z.data_ptr(), g.data_ptr())
+    ref = wl.grad(3, np.zeros(wl.d, np.float32))
+    assert np.array_equal(_np(g), ref) and 0.02 < (ref[:64 * 300] != 0).mean() < 0.25
+    sub = wl.device(j0=1000, n=7777)
+    gs = torch.empty(7777, dtype=torch.float32, device="cuda")
+    sub.grad_ptr(3, z.data_ptr(), gs.data_ptr())
+    assert np.array_equal(_np(gs), ref[1000:8777])
+
+
+# ----------------------------------------------------------------------------- small, exhaustive
+@pytest.mark.parametrize("variant", ["GA", "SA", "ASGD"])
+@pytest.mark.parametrize("window", [1, 4, 16])
+def test_mini_trajectory(P, variant, window):
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("mini")
+    for c_order in ((0, 1) if variant == "GA" else (0,)):
+        run = Run(wl, variant, window, options={P.GA_OPT_C_ORDER: c_order})
+        delays = run.run()
+        o, odelays, _ = run_oracle(wl, variant, c_order=c_order)
+        assert delays == odelays
+        _compare_engine(P, run, o, label=f"{variant}/c_order={c_order}/K={window}: ")
+        for i in range(wl.n_workers):
+            assert _same(_np(run.engine.saved(i)), o.saved(i))
+            assert run.engine.worker_iter(i) == o.iter(i)
+        run.close()
+
+
+@pytest.mark.parametrize("d", [1, 3, 4, 5, 31, 33, 255, 1025])
+def test_ragged_sizes(P, d):
+    from paper_1909_10802_b200.runner import Run
+    wl = W.Workload(name=f"d{d}", segments=[d], n_workers=3, arrivals=20, schedule_kind="ticks", seed=100 + d)
+    run = Run(wl, "GA", 16)
+    delays = run.run()
+    o, odelays, _ = run_oracle(wl, "GA")
+    assert delays == odelays
+    _compare_engine(P, run, o)
+    run.close()
+
+
+# ----------------------------------------------------------------------------- the five workloads
+def test_c1_full_with_checkpoints(P):
+    """C1 (ResNet-20 shape, 8 workers, 1000 arrivals), every element, 3 checkpoints + the end."""
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("C1")
+    cps = (250, 500, 750)
+    o, odelays, snaps = run_oracle(wl, "GA", checkpoints=cps)
+    run = Run(wl, "GA", 16)
+    for cp in cps:
+        run.run(cp)
+        for which, ref in zip((P.GA_THETA, P.GA_V, P.GA_M), snaps[cp]):
+            got = _np(run.engine.get(which))
+            assert _close(got, ref) and _same(got, ref), f"checkpoint {cp}, vector {which}"
+    run.run()
+    assert run.delays == odelays
+    _compare_engine(P, run, o)
+    run.close()
+
+
+def _sampled(P, name, variant, window, n_sample=4096, n_arrivals=None, options=None):
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config(name)
+    idx = wl.sample_indices(n_sample)
+    run = Run(wl, variant, window, options=options)
+    run.run(n_arrivals)
+    o, odelays, _ = run_oracle(wl, variant, n_arrivals=n_arrivals, idx=idx)
+    assert run.delays == odelays, "delays must be identical integers"
+    _compare_engine(P, run, o, idx=idx, label=f"{name}/{variant}/K={window}: ")
+    return run
+
+
+@pytest.mark.parametrize("variant", ["GA", "SA", "ASGD"])
+def test_c2_heterogeneous_workers(P, variant):
+    _sampled(P, "C2", variant, 16).close()
+
+
+def test_c3_window_invariance(P):
+    """ResNet-50 shape: K = 1, 4, 16 all match the oracle and each other, bit for bit."""
+    import torch
+    ref = None
+    for window in (16, 4, 1):
+        run = _sampled(P, "C3", "GA", window, n_arrivals=2000 if window == 16 else 300)
+        if window != 16:
+            full = [run.engine.get(w).clone() for w in (P.GA_THETA, P.GA_V, P.GA_M)]
+            if ref is None:
+                ref = full
+            else:
+                assert all(torch.equal(a, b) for a, b in zip(ref, full)), "K=1 and K=4 disagree"
+        run.close()
+        torch.cuda.empty_cache()
+
+
+def test_c4_stragglers(P):
+    import torch
+    _sampled(P, "C4", "GA", 16).close()
+    torch.cuda.empty_cache()
+
+
+def test_c5_transformer_lm_full_size(P):
+    """The benchmark configuration itself: 150M parameters, 32 saved copies, K = 16."""
+    import torch
+    _sampled(P, "C5", "GA", 16).close()
+    torch.cuda.empty_cache()
+
+
+# ----------------------------------------------------------------------------- single calls
+def _small_engine(P, d=5003, n=4, variant=None, seed=5):
+    import torch
+    rng = np.random.default_rng(seed)
+    th0 = rng.normal(size=d).astype(np.float32)
+    eng = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA if variant is None else variant)
+    eng.set_params(torch.from_numpy(th0).cuda())
+    o = oracle.Oracle(d, n, 0.1, 0.9, 0.999, variant if variant is not None else oracle.GA)
+    o.set_params(th0)
+    return eng, o, rng
+
+
+def test_push_then_pull_equals_batch_of_one(P):
+    """ga_push + ga_pull (TMA bulk copy) as separate calls, including a second push without
+    a pull in between."""
+    import torch
+    eng, o, rng = _small_engine(P)
+    for step, i in enumerate([0, 1, 1, 2, 0, 3, 3]):
+        g = rng.normal(size=eng.n_params).astype(np.float32)
+        assert eng.push(i, torch.from_numpy(g).cuda()) == o.push(i, g)
+        if step != 1:
+            sent = eng.pull(i)
+            o.pull(i)
+            assert _same(_np(sent), o.saved(i))
+    for which, ow in ((P.GA_THETA, o.THETA), (P.GA_V, o.V), (P.GA_M, o.M), (P.GA_C, o.C)):
+        assert _same(_np(eng.get(which)), o.get(ow))
+    for i in range(4):
+        assert _same(_np(eng.saved(i)), o.saved(i)) and eng.worker_iter(i) == o.iter(i)
+        assert _same(_np(eng.gap(i)), o.gap(i))
+    eng.close()
+
+
+def test_pull_bulk_copy_large(P):
+    """A pull of a vector spanning many 16 KB bulk copies and a ragged last one."""
+    import torch
+    d = 3_000_017
+    eng = P.Engine(d, 2, 0.1, 0.9, 0.999, P.GA_ASGD)
+    th0 = torch.randn(d, device="cuda")
+    eng.set_params(th0)
+    g = torch.randn(d, device="cuda")
+    eng.push(0, g)
+    sent = eng.pull(1)
+    assert torch.equal(sent, eng.get(P.GA_THETA)) and torch.equal(eng.saved(0), th0)
+    eng.close()
+
+
+def test_batch_with_repeated_workers_and_empty_batch(P):
+    import torch
+    eng, o, rng = _small_engine(P, n=3)
+    sched = [0, 1, 0, 0, 2, 1, 2, 2]
+    grads = [rng.normal(size=eng.n_params).astype(np.float32) for _ in sched]
+    delays, launches = eng.push_batch(sched, [torch.from_numpy(g).cuda() for g in grads], return_launches=True)
+    assert delays == o.push_batch(sched, grads)
+    assert launches == len(W.windows(sched, 16)) == 5
+    assert eng.push_batch([], []) == []
+    for which, ow in ((P.GA_THETA, o.THETA), (P.GA_V, o.V), (P.GA_M, o.M)):
+        assert _same(_np(eng.get(which)), o.get(ow))
+    eng.close()
+
+
+def test_gap_statistics(P):
+    import torch
+    eng, o, rng = _small_engine(P, d=70001, n=3)
+    eng.set_option(P.GA_OPT_STATS, 1)
+    with pytest.raises(P.GaError):
+        eng.get_stats()
+    sched = [0, 1, 2, 1, 0]
+    grads = [rng.normal(size=eng.n_params).astype(np.float32) for _ in sched]
+    dev = [torch.from_numpy(g).cuda() for g in grads]
+    for j, (i, g) in enumerate(zip(sched, grads)):          # one arrival at a time
+        eng.push_batch([i], [dev[j]])
+        o.push(i, g)
+        o.pull(i)
+        s, m = eng.get_stats()
+        os_, om = o.stats()
+        assert abs(s - os_) <= 1e-9 * os_ and m == om
+    # a fused window reports the statistics of its last arrival
+    eng.push_batch([0, 1, 2], dev[:3])
+    o.push_batch([0, 1, 2], grads[:3])
+    s, m = eng.get_stats()
+    assert abs(s - o.stats()[0]) <= 1e-9 * o.stats()[0] and m == o.stats()[1]
+    assert _same(_np(eng.get(P.GA_THETA)), o.get(o.THETA))
+    eng.close()
+
+
+def test_checkpoint_resume_is_bit_identical(P):
+    from paper_1909_10802_b200.runner import Run
+    import torch
+    wl = W.config("mini")
+    a = Run(wl, "GA", 4)
+    a.run(30)
+    blob = a.engine.export_state()
+    b = Run(wl, "GA", 4)
+    b.engine.import_state(blob)
+    b.k = 30
+    a.run()
+    b.run()
+    for which in (P.GA_THETA, P.GA_V, P.GA_M, P.GA_C):
+        assert torch.equal(a.engine.get(which), b.engine.get(which))
+    assert a.delays[30:] == b.delays
+    st = P.unpack_state(blob)
+    assert st["k_done"] == 30 and P.pack_state(st) == blob
+    with pytest.raises(P.GaError):
+        b.engine.import_state(blob[:100])
+    a.close()
+    b.close()
+
+
+def test_host_buffer_path_equals_device_path(P):
+    import torch
+    d, n = 9_000_011, 3      # three chunks of the host path, ragged end
+    rng = np.random.default_rng(3)
+    th0 = torch.from_numpy(rng.normal(size=d).astype(np.float32)).cuda()
+    sched = [2, 0, 1, 0]
+    grads = [torch.from_numpy(rng.normal(size=d).astype(np.float32)).pin_memory() for _ in sched]
+    outs = [torch.empty(d, dtype=torch.float32).pin_memory() for _ in sched]
+    a = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA)
+    b = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA)
+    a.set_params(th0)
+    b.set_params(th0)
+    da, _ = a.push_batch_host(sched, grads, outs)
+    sent_dev = []
+    db = []
+    for i, g in zip(sched, grads):
+        db += b.push_batch([i], [g.cuda()])
+        sent_dev.append(b.saved(i).clone())
+    assert da == db
+    for which in (P.GA_THETA, P.GA_V, P.GA_M):
+        assert torch.equal(a.get(which), b.get(which))
+    for o_host, s_dev in zip(outs, sent_dev):
+        assert torch.equal(o_host.cuda(), s_dev)
+    a.close()
+    b.close()
+
+
+# ----------------------------------------------------------------------------- fp64 and fast mode
+@pytest.mark.parametrize("math_mode", [0, 1])
+def test_single_arrival_against_fp64(P, math_mode):
+    """From one fp32 state, one arrival on the GPU (exact or fast math) and in the fp64 oracle."""
+    import torch
+    wl = W.config("C1")
+    idx = wl.sample_indices(20000)
+    d = len(idx)
+    sched = wl.schedule()
+    for start in (0, 40, 300):
+        o32, _, _ = run_oracle(wl, "GA", n_arrivals=start, idx=idx)
+        th, v, m, saved, iters, k_done, k_c = o32.state()
+        o64 = oracle.Oracle(d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, oracle.GA, precision=64)
+        o64.set_state(th, v, m, saved, iters, k_done, k_c)
+        eng = P.Engine(d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, P.GA_GA)
+        eng.set_option(P.GA_OPT_MATH, math_mode)
+        st = P.unpack_state(eng.export_state())
+        st.update(theta=th, v=v, m=m, saved=saved, iter=iters, k_done=k_done, k_c=k_c)
+        eng.import_state(P.pack_state(st))
+        i = sched[start]
+        g = wl.grad(start + 1, o32.sent_f32(i), idx)
+        assert eng.push_batch([i], [torch.from_numpy(g).cuda()]) == [o64.push(i, g)]
+        o64.pull(i)
+        for which, ow in ((P.GA_THETA, o64.THETA), (P.GA_V, o64.V), (P.GA_M, o64.M)):
+            got, ref = _np(eng.get(which)), o64.get(ow)
+            assert within(got, ref, TOL), (start, which, worst(got, ref))
+        eng.close()
+
+
+# ----------------------------------------------------------------------------- errors
+def test_bad_arguments_return_errors(P):
+    import ctypes
+    import torch
+    l = P.lib()
+    assert not l.ga_create(0, 4, 0.1, 0.9, 0.999, P.GA_GA) and "n_params" in P.last_error()
+    assert not l.ga_create(10, 0, 0.1, 0.9, 0.999, P.GA_GA)
+    assert not l.ga_create(10, 4, -1.0, 0.9, 0.999, P.GA_GA)
+    assert not l.ga_create(10, 4, 0.1, 1.0, 0.999, P.GA_GA)
+    assert not l.ga_create(10, 4, 0.1, 0.9, 1.0, P.GA_GA)
+    assert not l.ga_create(10, 4, 0.1, 0.9, 0.999, 7)
+    assert l.ga_push(None, 0, None) == P.GA_ERR_ARG
+    l.ga_destroy(None)
+    eng = P.Engine(1000, 4, 0.1, -0.5, 0.999, P.GA_GA)     # negative momentum is legal
+    g = torch.zeros(1004, device="cuda")
+    h = eng._h
+    assert l.ga_push(h, 4, g.data_ptr()) == P.GA_ERR_ARG and "worker" in P.last_error()
+    assert l.ga_push(h, -1, g.data_ptr()) == P.GA_ERR_ARG
+    assert l.ga_push(h, 0, None) == P.GA_ERR_ARG
+    assert l.ga_push(h, 0, g.data_ptr() + 4) == P.GA_ERR_ARG and "aligned" in P.last_error()
+    assert not l.ga_pull(h, 99)
+    assert l.ga_set_option(h, 99, 1.0) == P.GA_ERR_ARG
+    assert l.ga_set_option(h, P.GA_OPT_WINDOW, 17.0) == P.GA_ERR_ARG
+    sched = (ctypes.c_int * 2)(0, 9)
+    ptrs = (ctypes.c_void_p * 2)(g.data_ptr(), g.data_ptr())
+    assert l.ga_push_batch(h, sched, ptrs, 2, None) == P.GA_ERR_ARG
+    assert eng.num_arrivals == 0, "a rejected batch applies nothing"
+    assert l.ga_push_batch(h, sched, ptrs, -1, None) == P.GA_ERR_ARG
+    assert eng.push(0, g) == 1 and eng.num_arrivals == 1     # still usable
+    assert l.ga_set_option(h, P.GA_OPT_C_ORDER, 1.0) == P.GA_ERR_STATE
+    eng.close()
+
+
+def test_non_finite_gradient_propagates(P):
+    import torch
+    eng, o, rng = _small_engine(P, d=257, n=2)
+    g = rng.normal(size=257).astype(np.float32)
+    g[3], g[100], g[200] = np.nan, np.inf, -np.inf
+    assert eng.push_batch([0], [torch.from_numpy(g).cuda()]) == o.push_batch([0], [g])
+    g2 = rng.normal(size=257).astype(np.float32)
+    assert eng.push_batch([1], [torch.from_numpy(g2).cuda()]) == o.push_batch([1], [g2])
+    for which, ow in ((P.GA_THETA, o.THETA), (P.GA_V, o.V), (P.GA_M, o.M)):
+        assert _same(_np(eng.get(which)), o.get(ow))
+    eng.close()

@@ -232,10 +232,10 @@ def cuda_lib():
         l = ctypes.CDLL(_CUDA_LIB)
         c = ctypes
         l.wl_cuda_init.restype = c.c_int
-        l.wl_cuda_init.argtypes = [c.c_uint64, c.c_int64, c.c_void_p, c.c_void_p]
+        l.wl_cuda_init.argtypes = [c.c_uint64, c.c_int64, c.c_int64, c.c_void_p, c.c_void_p]
         l.wl_cuda_grad.restype = c.c_int
-        l.wl_cuda_grad.argtypes = [c.POINTER(_Spec), c.c_void_p, c.c_void_p, c.c_int64, c.c_void_p,
-                                   c.c_void_p, c.c_void_p]
+        l.wl_cuda_grad.argtypes = [c.POINTER(_Spec), c.c_void_p, c.c_void_p, c.c_int64, c.c_int64,
+                                   c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p]
         _cuda = l
     return _cuda
 
@@ -275,20 +275,26 @@ class Workload:
                           self.emb_rows * self.emb_row, max(self.emb_row, 1), thresh)
 
     # -- host-side inputs
-    def schedule(self):
+    def schedule(self, arrivals=None):
+        """The workload's arrival schedule; `arrivals` asks for a longer (or shorter) run of
+        the same simulation (the first self.arrivals entries are the workload's own)."""
+        if arrivals is not None:
+            return self._simulate(arrivals)
         if self._sched is None:
-            kind, n, a = self.schedule_kind, self.n_workers, self.arrivals
-            if kind == "ticks":
-                self._sched = schedule_uniform_ticks(self.seed, n, a)
-            elif kind == "lognormal":
-                self._sched = schedule_lognormal(self.seed, n, a)
-            elif kind == "exp_stragglers":
-                self._sched = schedule_exponential_stragglers(self.seed, n, a)
-            elif kind == "round_robin":
-                self._sched = schedule_round_robin(n, a)
-            else:
-                raise ValueError(kind)
+            self._sched = self._simulate(self.arrivals)
         return self._sched
+
+    def _simulate(self, a):
+        kind, n = self.schedule_kind, self.n_workers
+        if kind == "ticks":
+            return schedule_uniform_ticks(self.seed, n, a)
+        if kind == "lognormal":
+            return schedule_lognormal(self.seed, n, a)
+        if kind == "exp_stragglers":
+            return schedule_exponential_stragglers(self.seed, n, a)
+        if kind == "round_robin":
+            return schedule_round_robin(n, a)
+        raise ValueError(kind)
 
     def sample_indices(self, n, extra_seed=0):
         """Global element indices for a sampled parity check: both ends of every segment,
@@ -336,16 +342,19 @@ class Workload:
         return out
 
     # -- device generators
-    def device(self, torch_device="cuda"):
-        return DeviceWorkload(self, torch_device)
+    def device(self, torch_device="cuda", j0=0, n=None):
+        return DeviceWorkload(self, torch_device, j0, n)
 
 
 class DeviceWorkload:
     """Device-side twin of Workload's generators (torch only holds the memory)."""
 
-    def __init__(self, wl, torch_device):
+    def __init__(self, wl, torch_device, j0=0, n=None):
         import torch
         self.wl = wl
+        self.j0 = int(j0)                                  # this holder covers [j0, j0 + n)
+        self.n = int(wl.d - j0 if n is None else n)
+        assert 0 <= self.j0 and self.j0 + self.n <= wl.d
         self._torch = torch
         self.seg_off = torch.from_numpy(wl.seg_off).to(torch_device)
         self.seg_sigma = torch.from_numpy(wl.seg_sigma).to(torch_device)
@@ -355,15 +364,15 @@ class DeviceWorkload:
         return ctypes.c_void_p(self._torch.cuda.current_stream().cuda_stream)
 
     def theta0(self, out):
-        assert out.dtype == self._torch.float32 and out.numel() >= self.wl.d and out.is_contiguous()
-        rc = self.lib.wl_cuda_init(self.wl.seed, self.wl.d, ctypes.c_void_p(out.data_ptr()), self._stream())
+        assert out.dtype == self._torch.float32 and out.numel() >= self.n and out.is_contiguous()
+        rc = self.lib.wl_cuda_init(self.wl.seed, self.j0, self.n, ctypes.c_void_p(out.data_ptr()), self._stream())
         if rc:
             raise RuntimeError(f"wl_cuda_init: CUDA error {rc}")
         return out
 
     def grad_ptr(self, k, sent_ptr, out_ptr):
         rc = self.lib.wl_cuda_grad(ctypes.byref(self.wl.spec), ctypes.c_void_p(self.seg_off.data_ptr()),
-                                   ctypes.c_void_p(self.seg_sigma.data_ptr()), k,
+                                   ctypes.c_void_p(self.seg_sigma.data_ptr()), k, self.j0, self.n,
                                    ctypes.c_void_p(sent_ptr), ctypes.c_void_p(out_ptr), self._stream())
         if rc:
             raise RuntimeError(f"wl_cuda_grad: CUDA error {rc}")
