@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C5")
+    ap.add_argument("--params", type=int, default=0, help="profiling aid: a one-segment vector of this size")
+    ap.add_argument("--workers", type=int, default=32)
     ap.add_argument("--variant", default="GA", choices=["GA", "SA", "ASGD"])
     ap.add_argument("--window", type=int, default=16)
     ap.add_argument("--math", default="exact", choices=["exact", "fast"])
@@ -122,6 +124,14 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def pick_workload(args):
+    import workloads as W
+    if args.params:
+        return W.Workload(name=f"custom{args.params}", segments=[args.params], n_workers=args.workers,
+                          arrivals=500, schedule_kind="ticks", seed=W.BASE_SEED + 99)
+    return W.config(args.config)
+
+
 def bench_windows(wl, window, count):
     """`count` windows of the workload's schedule (the simulation is run as long as needed)."""
     import workloads as W
@@ -165,7 +175,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = W.config(args.config)
+    wl = pick_workload(args)
     n_params = min(args.cpu_sample_params // 4, wl.d)
     wins = bench_windows(wl, args.window, args.steps + args.warmup)
     time_oracle(wl, args.variant, n_params, wins[:args.warmup])
@@ -202,7 +212,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     P.lib()
 
-    base = W.config(args.config)
+    base = pick_workload(args)
     # weak scaling: rank r owns the r-th C5-sized range of a world-times larger vector
     wl = base if world == 1 else W.Workload(
         **{**{f: getattr(base, f) for f in ("name", "segments", "n_workers", "arrivals", "schedule_kind", "lr",
