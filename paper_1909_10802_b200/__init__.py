@@ -13,7 +13,7 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libga.so")
+LIB_PATH = os.environ.get("GA_LIBRARY") or os.path.join(_HERE, "libga.so")   # GA_LIBRARY: another build
 
 GA_ASGD, GA_SA, GA_GA = 0, 1, 2
 GA_OK, GA_ERR_ARG, GA_ERR_STATE, GA_ERR_OOM, GA_ERR_CUDA = 0, -1, -2, -3, -4

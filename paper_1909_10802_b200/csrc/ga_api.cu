@@ -135,7 +135,7 @@ int grid_1d(long long n, int threads, int cap) {
 // ----------------------------------------------------------------------------- launch
 template <int VARIANT, bool EXACT, int C_ORDER, bool STATS>
 void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st) {
-    constexpr int B = 4;
+    constexpr int B = GA_WINDOW_BATCH;
     const long long nvec = vec_end - vec_begin;
     long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
