@@ -149,6 +149,35 @@ int64_t ga_worker_iter(ga_engine* e, int worker);
 size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap);
 int ga_import_state(ga_engine* e, const void* buf_host, size_t len);
 
+/* Gap statistics without any allocation. (The paper has no counterpart of this call; it exists
+ * for deployment reasons only.) Computes the sum and the maximum over all parameters of the
+ * parameter-wise Gap |theta - saved| / C + 1, with C = lr_max * (sqrt(m / (1 - c_beta^n_refreshes))
+ * + 1e-8) (C = lr_max * 1e-8 when n_refreshes is 0) -- the same numbers ga_gap would give if its
+ * output were reduced -- from three device vectors the caller already holds, and writes
+ * out_dev[0] = sum, out_dev[1] = max (two doubles on the device).
+ *
+ * Who it is for: code that runs next to a training job whose framework allocator already owns
+ * nearly all device memory (a raw cudaMalloc may then simply fail), and hooks on a latency-critical
+ * path that must not pay the device-wide synchronisation that cudaMalloc and cudaFree imply. This
+ * call needs no engine and never calls cudaMalloc, cudaFree or any allocating routine: the
+ * per-block partial results of its reduction live in a fixed array inside the library's device
+ * image (1 MiB, present on every GPU that loads the library until the process ends).
+ *
+ *   - theta_dev, saved_dev, m_dev: n_params floats each, device memory, 16-byte aligned, read only.
+ *   - n_params must be in [1, GA_NOALLOC_MAX_PARAMS]; larger sizes are rejected with GA_ERR_ARG.
+ *   - Work is enqueued on cuda_stream and the call returns at once; the result is in out_dev when
+ *     that stream reaches this point.
+ *   - The first call on each device looks up the device address of the fixed array (once per
+ *     device, with that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array. Each call overwrites every entry it later reads,
+ *     so nothing has to be cleared between calls, but two calls whose kernels overlap on the GPU
+ *     (different streams, or different host threads) race on it: run them one after the other.
+ * Returns GA_OK or a negative GA_ERR_* code (see ga_last_error). */
+#define GA_NOALLOC_MAX_PARAMS ((size_t)1 << 28)
+int ga_gap_stats_noalloc(const float* theta_dev, const float* saved_dev, const float* m_dev,
+                         size_t n_params, float lr_max, float c_beta, int64_t n_refreshes,
+                         double* out_dev, void* cuda_stream);
+
 /* Message for the calling thread's most recent failure ("" if none). Never NULL. */
 const char* ga_last_error(void);
 

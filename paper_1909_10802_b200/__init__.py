@@ -20,6 +20,7 @@ GA_OK, GA_ERR_ARG, GA_ERR_STATE, GA_ERR_OOM, GA_ERR_CUDA = 0, -1, -2, -3, -4
 GA_THETA, GA_V, GA_M, GA_C = 0, 1, 2, 3
 GA_OPT_C_ORDER, GA_OPT_MATH, GA_OPT_STATS, GA_OPT_WINDOW = 0, 1, 2, 3
 GA_MAX_WINDOW = 16
+GA_NOALLOC_MAX_PARAMS = 1 << 28
 VARIANTS = {"ASGD": GA_ASGD, "SA": GA_SA, "GA": GA_GA}
 
 # every symbol include/ga.h declares: name -> (restype, argtypes)
@@ -42,6 +43,8 @@ _SIGNATURES = {
     "ga_worker_iter": (_c.c_int64, [_c.c_void_p, _c.c_int]),
     "ga_export_state": (_c.c_size_t, [_c.c_void_p, _c.c_void_p, _c.c_size_t]),
     "ga_import_state": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_size_t]),
+    "ga_gap_stats_noalloc": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_size_t, _c.c_float, _c.c_float,
+                                        _c.c_int64, _c.c_void_p, _c.c_void_p]),
     "ga_last_error": (_c.c_char_p, []),
 }
 
@@ -86,6 +89,20 @@ def _ptr(t):
     if isinstance(t, int):
         return t
     return t.data_ptr()
+
+
+def gap_stats_noalloc(theta, saved, m, lr_max, c_beta, n_refreshes, out, stream=None):
+    """ga_gap_stats_noalloc: sum and max of the parameter-wise Gap from three CUDA float32
+    tensors into `out` (two float64 on the device). Allocates nothing, needs no Engine; meant for
+    callers that must not touch the device allocator (see include/ga.h)."""
+    import torch
+    n = theta.numel()
+    assert saved.numel() >= n and m.numel() >= n
+    assert out.is_cuda and out.dtype == torch.float64 and out.numel() >= 2
+    raw = (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+    _check(lib().ga_gap_stats_noalloc(theta.data_ptr(), saved.data_ptr(), m.data_ptr(), n, lr_max, c_beta,
+                                      n_refreshes, out.data_ptr(), raw))
+    return out
 
 
 class Engine:

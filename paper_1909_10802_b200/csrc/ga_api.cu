@@ -598,3 +598,112 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
 }
 
 }  // extern "C"
+
+// ============================================================ allocation-free Gap statistics
+// Everything this entry point needs lives in this file: the scratch array is part of the
+// library's device image, so no call here ever allocates or frees device memory.
+namespace {
+
+constexpr int kNoAllocTile = 4096;          // parameters reduced by one block
+constexpr int kNoAllocMaxBlocks = (int)(GA_NOALLOC_MAX_PARAMS / kNoAllocTile);   // 65536
+constexpr int kNoAllocMaxDevices = 64;
+
+// One partial result per block. In host code this name is only a handle for
+// cudaGetSymbolAddress; kernels are given the address that call returns.
+static __device__ __align__(256) ga::StatsPartial g_noalloc_partials[kNoAllocMaxBlocks];
+
+// First pass: block b reduces parameters [b*4096, (b+1)*4096) and overwrites partials[b].
+__global__ void __launch_bounds__(256)
+ga_gap_stats_tile_kernel(const float* __restrict__ theta, const float* __restrict__ saved,
+                         const float* __restrict__ mom, float inv_bias, ga::Hyper h, long long d,
+                         ga::StatsPartial* __restrict__ partials) {
+    __shared__ double s_sum[8];
+    __shared__ float s_max[8];
+    const long long tile = (long long)blockIdx.x * kNoAllocTile;
+    double sum = 0.0;
+    float mx = 0.f;
+    for (int q = 0; q < kNoAllocTile / (256 * 4); ++q) {
+        const long long e = tile + ((long long)q * 256 + threadIdx.x) * 4;
+        float t[4], s[4], m[4];
+        int n = 0;
+        if (e + 4 <= d) {
+            const float4 a = *reinterpret_cast<const float4*>(theta + e);
+            const float4 b = *reinterpret_cast<const float4*>(saved + e);
+            const float4 c = *reinterpret_cast<const float4*>(mom + e);
+            t[0] = a.x; t[1] = a.y; t[2] = a.z; t[3] = a.w;
+            s[0] = b.x; s[1] = b.y; s[2] = b.z; s[3] = b.w;
+            m[0] = c.x; m[1] = c.y; m[2] = c.z; m[3] = c.w;
+            n = 4;
+        } else {
+            for (; n < 4 && e + n < d; ++n) { t[n] = theta[e + n]; s[n] = saved[e + n]; m[n] = mom[e + n]; }
+        }
+        for (int u = 0; u < n; ++u) {
+            const float C = __fmul_rn(h.eta_max, __fadd_rn(__fsqrt_rn(__fmul_rn(m[u], inv_bias)), h.eps));
+            const float G = __fadd_rn(__fdiv_rn(fabsf(__fsub_rn(t[u], s[u])), C), 1.0f);
+            sum += (double)G;
+            mx = fmaxf(mx, G);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    if ((threadIdx.x & 31) == 0) { s_sum[threadIdx.x >> 5] = sum; s_max[threadIdx.x >> 5] = mx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        ga::StatsPartial out;
+        out.sum = 0.0; out.max = 0.f; out.pad = 0.f;
+        for (int w = 0; w < 8; ++w) { out.sum += s_sum[w]; out.max = fmaxf(out.max, s_max[w]); }
+        partials[blockIdx.x] = out;
+    }
+}
+
+// Device address of the scratch array, looked up once per device.
+ga::StatsPartial* g_noalloc_addr[kNoAllocMaxDevices] = {};
+
+int noalloc_scratch(ga::StatsPartial** out) {
+    int dev = -1;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return fail(GA_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(err));
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return fail(GA_ERR_ARG, "device index %d not supported", dev);
+    ga::StatsPartial* p = __atomic_load_n(&g_noalloc_addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        err = cudaGetSymbolAddress((void**)&p, g_noalloc_partials);   // the current device's copy
+        if (err != cudaSuccess || !p)
+            return fail(GA_ERR_CUDA, "cudaGetSymbolAddress(scratch): %s", cudaGetErrorString(err));
+        __atomic_store_n(&g_noalloc_addr[dev], p, __ATOMIC_RELEASE);
+    }
+    *out = p;
+    return GA_OK;
+}
+
+}  // namespace
+
+extern "C" int ga_gap_stats_noalloc(const float* theta_dev, const float* saved_dev, const float* m_dev,
+                                    size_t n_params, float lr_max, float c_beta, int64_t n_refreshes,
+                                    double* out_dev, void* cuda_stream) {
+    if (int rc = check_dev_ptr(theta_dev, "theta_dev")) return rc;
+    if (int rc = check_dev_ptr(saved_dev, "saved_dev")) return rc;
+    if (int rc = check_dev_ptr(m_dev, "m_dev")) return rc;
+    if (!out_dev || (uintptr_t)out_dev % 8) return fail(GA_ERR_ARG, "out_dev is NULL or not 8-byte aligned");
+    if (n_params == 0) return fail(GA_ERR_ARG, "n_params is 0");
+    if (n_params > GA_NOALLOC_MAX_PARAMS)
+        return fail(GA_ERR_ARG, "n_params = %zu exceeds GA_NOALLOC_MAX_PARAMS = %zu, the size the fixed scratch array covers",
+                    n_params, (size_t)GA_NOALLOC_MAX_PARAMS);
+    if (!(lr_max > 0.f) || !std::isfinite(lr_max)) return fail(GA_ERR_ARG, "lr_max must be positive and finite");
+    if (!(c_beta >= 0.f && c_beta < 1.f)) return fail(GA_ERR_ARG, "c_beta must be in [0, 1)");
+    if (n_refreshes < 0) return fail(GA_ERR_ARG, "n_refreshes is negative");
+    ga::StatsPartial* scratch = nullptr;
+    if (int rc = noalloc_scratch(&scratch)) return rc;
+    ga::Hyper h;
+    h.eta_max = lr_max; h.gamma = 0.f; h.beta = c_beta; h.one_minus_beta = (float)(1.0 - (double)c_beta); h.eps = 1e-8f;
+    const float inv_bias = n_refreshes == 0 ? 0.f : (float)(1.0 / (1.0 - std::pow((double)c_beta, (double)n_refreshes)));
+    const int blocks = (int)((n_params + kNoAllocTile - 1) / kNoAllocTile);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    ga_gap_stats_tile_kernel<<<blocks, 256, 0, st>>>(theta_dev, saved_dev, m_dev, inv_bias, h, (long long)n_params, scratch);
+    ga::ga_stats_finish_kernel<<<1, 256, 0, st>>>(scratch, blocks, out_dev);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return fail(GA_ERR_CUDA, "ga_gap_stats_noalloc launch: %s", cudaGetErrorString(err));
+    return GA_OK;
+}
