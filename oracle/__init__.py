@@ -21,7 +21,9 @@ def build(force=False, src=_SRC, out=_LIB):
     """Compile the oracle with g++ (no fast-math, no FMA contraction)."""
     if not force and os.path.exists(out) and os.path.getmtime(out) >= os.path.getmtime(src):
         return out
-    subprocess.check_call(["g++", *CXXFLAGS, "-o", out, src])
+    tmp = f"{out}.{os.getpid()}.tmp"          # several test workers may build at once
+    subprocess.check_call(["g++", *CXXFLAGS, "-o", tmp, src])
+    os.replace(tmp, out)
     return out
 
 

@@ -31,6 +31,8 @@
 //   * eta_max is the learning rate given at creation.
 //   * delay tau_k = k - iter[i], k counting arrivals from 1, iter[] starting at 0;
 //     a pull records the number of pushes applied so far.
+//   * The penalised gradient is formed as the algorithm prints it, (1/G_k) (.) g: the
+//     reciprocal of the Gap, rounded, then an elementwise product.
 //   * Arithmetic: every line below is one IEEE operation per symbol, in the order
 //     written, with v <- gamma*v + g_hat and theta <- theta - eta*v each a single fused
 //     multiply-add. Build with -ffp-contract=off so nothing else is fused.
@@ -132,7 +134,8 @@ struct Master {
                 const T C = coeff(m[j], ib);
                 const T dist = std::fabs(theta[j] - s[j]);
                 const T G = dist / C + (T)1;
-                const T g_hat = g / G;
+                const T inv_gap = (T)1 / G;       // the printed form: (1/G_k) (.) g
+                const T g_hat = inv_gap * g;
                 v[j] = std::fma(gamma, v[j], g_hat);
                 theta[j] = std::fma(-eta, v[j], theta[j]);
                 sum_gap += (double)G;

@@ -16,7 +16,8 @@ SRC = os.path.join(os.path.dirname(oracle.__file__), "ga_oracle.cpp")
 # (name, text in the oracle, replacement)
 MUTANTS = [
     ("gap_without_plus_one", "const T G = dist / C + (T)1;", "const T G = dist / C;"),
-    ("gap_multiplies_gradient", "const T g_hat = g / G;", "const T g_hat = g * G;"),
+    ("gap_multiplies_gradient", "const T inv_gap = (T)1 / G;", "const T inv_gap = G;"),
+    ("gap_reciprocal_unused", "const T g_hat = inv_gap * g;", "const T g_hat = g;"),
     ("gap_divides_by_C_squared", "const T G = dist / C + (T)1;", "const T G = dist / C / C + (T)1;"),
     ("gap_uses_signed_distance", "const T dist = std::fabs(theta[j] - s[j]);\n                const T G",
      "const T dist = theta[j] - s[j];\n                const T G"),

@@ -182,8 +182,10 @@ def build_cpu(force=False):
     if not force and os.path.exists(_CPU_LIB) and all(
             os.path.getmtime(_CPU_LIB) >= os.path.getmtime(s) for s in srcs):
         return _CPU_LIB
+    tmp = f"{_CPU_LIB}.{os.getpid()}.tmp"
     subprocess.check_call(["gcc", "-std=c11", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-Wall",
-                           "-o", _CPU_LIB, srcs[0], "-lm"])
+                           "-o", tmp, srcs[0], "-lm"])
+    os.replace(tmp, _CPU_LIB)
     return _CPU_LIB
 
 
@@ -192,9 +194,11 @@ def build_cuda(force=False):
     if not force and os.path.exists(_CUDA_LIB) and all(
             os.path.getmtime(_CUDA_LIB) >= os.path.getmtime(s) for s in srcs):
         return _CUDA_LIB
+    tmp = f"{_CUDA_LIB}.{os.getpid()}.tmp"
     subprocess.check_call(["nvcc", "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a",
                            "-lineinfo", "-fmad=false", "-Xcompiler", "-fPIC", "-shared",
-                           "-o", _CUDA_LIB, srcs[0]])
+                           "-o", tmp, srcs[0]])
+    os.replace(tmp, _CUDA_LIB)
     return _CUDA_LIB
 
 
