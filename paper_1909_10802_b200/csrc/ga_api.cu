@@ -135,12 +135,16 @@ int grid_1d(long long n, int threads, int cap) {
 // ----------------------------------------------------------------------------- launch
 template <int VARIANT, bool EXACT, int C_ORDER, bool STATS>
 void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st) {
-    constexpr int B = GA_WINDOW_BATCH;
     const long long nvec = vec_end - vec_begin;
     long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
-    ga::ga_window_kernel<VARIANT, EXACT, C_ORDER, STATS, B><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
-        e->theta, e->vel, e->mom, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
+    // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner
+    if (w.K == 1)
+        ga::ga_window_kernel<VARIANT, EXACT, C_ORDER, STATS, 1><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
+            e->theta, e->vel, e->mom, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
+    else
+        ga::ga_window_kernel<VARIANT, EXACT, C_ORDER, STATS, GA_WINDOW_BATCH><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
+            e->theta, e->vel, e->mom, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
     if (STATS) {
         ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev);
     }
