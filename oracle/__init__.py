@@ -13,7 +13,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ga_oracle.cpp")
 _LIB = os.path.join(_HERE, "libga_oracle.so")
 
-ASGD, SA, GA = 0, 1, 2
+ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA = range(7)
+VARIANTS = {"ASGD": ASGD, "SA": SA, "GA": GA, "SA_GRAD": SA_GRAD, "DANA": DANA, "DANA_SA": DANA_SA,
+            "DANA_GA": DANA_GA}
 CXXFLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-Wall", "-Wextra"]
 
 
@@ -44,7 +46,8 @@ def _bind(path):
     lib.gao_k_done.argtypes = [c.c_void_p]
     lib.gao_iter.restype = c.c_int64
     lib.gao_iter.argtypes = [c.c_void_p, c.c_int]
-    lib.gao_set_state.argtypes = [c.c_void_p] * 6 + [c.c_int64, c.c_int64]
+    lib.gao_set_state.argtypes = [c.c_void_p] * 6 + [c.c_int64, c.c_int64, c.c_void_p]
+    lib.gao_set_dana_sum.argtypes = [c.c_void_p, c.c_int]
     lib.gao_k_c.restype = c.c_int64
     lib.gao_k_c.argtypes = [c.c_void_p]
     lib.gao_stats.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
@@ -76,13 +79,15 @@ class Oracle:
     THETA, V, M, C = 0, 1, 2, 3
 
     def __init__(self, n_params, n_workers, lr, momentum, c_beta, variant, precision=32,
-                 c_order=0, eps=None, _lib=None):
+                 c_order=0, eps=None, dana_sum=1, _lib=None):
         self._l = _lib if _lib is not None else lib()
         self.d, self.n = int(n_params), int(n_workers)
         self._h = self._l.gao_create(self.d, self.n, lr, momentum, c_beta, variant, precision)
         if not self._h:
             raise ValueError("gao_create failed")
+        self.variant = variant
         self._l.gao_set_c_order(self._h, c_order)
+        self._l.gao_set_dana_sum(self._h, dana_sum)
         if eps is not None:
             self._l.gao_set_eps(self._h, eps)
 
@@ -123,6 +128,14 @@ class Oracle:
     def saved(self, worker):
         return self.get(4 + worker)
 
+    def worker_momentum(self, worker):
+        """DANA: v^worker."""
+        return self.get(100000 + worker)
+
+    @property
+    def is_dana(self):
+        return self.variant in (DANA, DANA_SA, DANA_GA)
+
     def sent_f32(self, worker):
         out = np.empty(self.d, dtype=np.float32)
         self._l.gao_sent_f32(self._h, worker, out.ctypes.data)
@@ -142,14 +155,22 @@ class Oracle:
         """(theta, v, m, saved[N][d], iter[N], k_done, k_c); vectors as float64."""
         saved = np.stack([self.saved(i) for i in range(self.n)])
         iters = np.asarray([self.iter(i) for i in range(self.n)], dtype=np.int64)
-        return (self.get(self.THETA), self.get(self.V), self.get(self.M), saved, iters,
-                self.k_done, int(self._l.gao_k_c(self._h)))
+        out = (self.get(self.THETA), self.get(self.V), self.get(self.M), saved, iters,
+               self.k_done, int(self._l.gao_k_c(self._h)))
+        if self.is_dana:
+            out += (np.stack([self.worker_momentum(i) for i in range(self.n)]),)
+        return out
 
-    def set_state(self, theta, v, m, saved, iters, k_done, k_c):
+    def set_state(self, theta, v, m, saved, iters, k_done, k_c, v_workers=None):
         a = [np.ascontiguousarray(x, dtype=np.float64) for x in (theta, v, m, saved)]
         assert a[0].shape == (self.d,) and a[3].shape == (self.n, self.d)
         it = np.ascontiguousarray(iters, dtype=np.int64)
-        self._l.gao_set_state(self._h, *(x.ctypes.data for x in a), it.ctypes.data, k_done, k_c)
+        vw = None
+        if self.is_dana:
+            vw = np.ascontiguousarray(v_workers, dtype=np.float64)
+            assert vw.shape == (self.n, self.d)
+        self._l.gao_set_state(self._h, *(x.ctypes.data for x in a), it.ctypes.data, k_done, k_c,
+                              None if vw is None else vw.ctypes.data)
 
     @property
     def k_done(self):

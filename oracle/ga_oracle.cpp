@@ -17,6 +17,11 @@
 //                        parameters" of the three master algorithms; the saved copy is
 //                        the theta^i = theta_{k-tau_k} of the appendix's remark
 //   momentum           : Section 3, the variant without dampening: v <- gamma v + g
+//   push, SA_GRAD      : Algorithm "Staleness-Aware-Gradient: master" (appendix): g / tau
+//   push/pull, DANA*   : Algorithms "DANA: master", "DANA-Staleness-Aware: master" and
+//                        "DANA-Gap-Aware: master" (appendix): one momentum vector v^i per
+//                        worker, theta <- theta - eta v^i, and the worker is sent (and, for
+//                        the Gap, the master saves) the estimate theta - eta gamma sum_j v^j
 //
 // Readings taken where the paper leaves a choice (all also listed in the design notes):
 //   * Order of C and Gap (option c_order). 0 = "lagged": the Gap at arrival k uses the C
@@ -33,6 +38,10 @@
 //     a pull records the number of pushes applied so far.
 //   * The penalised gradient is formed as the algorithm prints it, (1/G_k) (.) g: the
 //     reciprocal of the Gap, rounded, then an elementwise product.
+//   * DANA's sum over the workers' momentum vectors (option dana_sum): 1 = kept as a running
+//     sum, S <- (S - v^i_old) + v^i_new at each arrival (what a master would do; default);
+//     0 = the printed sum_{j=1..N} v^j evaluated afresh, in order, at every send. The two are
+//     equal in exact arithmetic and are pinned against each other.
 //   * Arithmetic: every line below is one IEEE operation per symbol, in the order
 //     written, with v <- gamma*v + g_hat and theta <- theta - eta*v each a single fused
 //     multiply-add. Build with -ffp-contract=off so nothing else is fused.
@@ -44,6 +53,7 @@
 // "parity unpinned": the choice between the two c_order readings and the value of C
 // before the first refresh -- nothing the paper prints separates them.
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -52,7 +62,7 @@
 
 namespace {
 
-enum Variant { ASGD = 0, SA = 1, GA = 2 };
+enum Variant { ASGD = 0, SA = 1, GA = 2, SA_GRAD = 3, DANA = 4, DANA_SA = 5, DANA_GA = 6 };
 
 template <typename T>
 struct Master {
@@ -67,6 +77,9 @@ struct Master {
     int c_order = 0;  // 0 lagged, 1 Adam order
     std::vector<T> theta, v, m;
     std::vector<T> saved;       // N x d, row i = theta^i, the parameters last sent to worker i
+    std::vector<T> vw;          // DANA: N x d, row i = v^i, worker i's momentum
+    std::vector<T> vsum;        // DANA: sum_j v^j
+    int dana_sum = 1;           // 1 running sum, 0 summed afresh at every send
     std::vector<int64_t> iter;  // iteration array of the SA algorithm
     int64_t k_done = 0;         // arrivals applied so far
     int64_t k_c = 0;            // refreshes of m so far
@@ -93,18 +106,89 @@ struct Master {
         for (int i = 0; i < n_workers; ++i) iter[i] = 0;
         k_done = 0;
         k_c = 0;
+        std::fill(vw.begin(), vw.end(), (T)0);
+        std::fill(vsum.begin(), vsum.end(), (T)0);
     }
 
+    bool is_dana() const { return variant == DANA || variant == DANA_SA || variant == DANA_GA; }
+    bool has_gap() const { return variant == GA || variant == DANA_GA; }
+
     void pull(int i) {
+        if (is_dana()) { pull_dana(i); return; }
         for (int64_t j = 0; j < d; ++j) saved[(size_t)i * d + j] = theta[j];
         iter[i] = k_done;
+    }
+
+    // DANA: "Send estimate theta_hat = theta - eta gamma sum_j v^j to worker i" (and save it).
+    void pull_dana(int i) {
+        const T eta_gamma = eta * gamma;
+        for (int64_t j = 0; j < d; ++j) {
+            T total = vsum[j];
+            if (dana_sum == 0) {
+                total = 0;
+                for (int w = 0; w < n_workers; ++w) total = total + vw[(size_t)w * d + j];
+            }
+            saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);
+        }
+        iter[i] = k_done;
+    }
+
+    // One arrival of the three DANA masters.
+    void push_dana(int i, const float* grad, int64_t tau) {
+        T* vi = &vw[(size_t)i * d];
+        const T* s = &saved[(size_t)i * d];
+        const T one_minus_beta = (T)(1.0 - (double)beta);
+        double sum_gap = 0.0, max_gap = 0.0;
+        if (variant == DANA_GA && c_order == 1) {
+            for (int64_t j = 0; j < d; ++j) {
+                const T u = std::fma(gamma, vi[j], (T)grad[j]);
+                m[j] = std::fma(beta, m[j], one_minus_beta * (u * u));
+            }
+            k_c += 1;
+        }
+        const T ib = k_c > 0 ? inv_bias() : (T)0;
+        for (int64_t j = 0; j < d; ++j) {
+            const T g = (T)grad[j];
+            T g_pen = g;                                   // DANA: the gradient as it is
+            if (variant == DANA_SA) {
+                g_pen = g / (T)tau;                        // DANA-SA: g / tau
+            } else if (variant == DANA_GA) {
+                const T C = coeff(m[j], ib);
+                const T dist = std::fabs(theta[j] - s[j]); // s = the estimate saved when sent
+                const T G = dist / C + (T)1;
+                const T inv_gap = (T)1 / G;
+                g_pen = inv_gap * g;
+                sum_gap += (double)G;
+                if ((double)G > max_gap) max_gap = (double)G;
+            }
+            const T v_old = vi[j];
+            const T v_new = std::fma(gamma, v_old, g_pen); // worker's momentum v^i
+            vi[j] = v_new;
+            theta[j] = std::fma(-eta, v_new, theta[j]);    // master's weights
+            vsum[j] = (vsum[j] - v_old) + v_new;           // running sum_j v^j
+        }
+        if (variant == DANA_GA && c_order == 0) {
+            for (int64_t j = 0; j < d; ++j)
+                m[j] = std::fma(beta, m[j], one_minus_beta * (vi[j] * vi[j]));
+            k_c += 1;
+        }
+        last_sum_gap = sum_gap;
+        last_max_gap = max_gap;
     }
 
     int64_t push(int i, const float* grad) {
         const int64_t k = k_done + 1;
         const int64_t tau = k - iter[i];
         const T* s = &saved[(size_t)i * d];
-        if (variant == ASGD) {
+        if (is_dana()) {
+            push_dana(i, grad, tau);
+        } else if (variant == SA_GRAD) {
+            for (int64_t j = 0; j < d; ++j) {
+                const T g_tau = (T)grad[j] / (T)tau;
+                v[j] = std::fma(gamma, v[j], g_tau);
+                theta[j] = std::fma(-eta, v[j], theta[j]);
+            }
+        } else if (variant == ASGD) {
             for (int64_t j = 0; j < d; ++j) {
                 const T g = (T)grad[j];
                 v[j] = std::fma(gamma, v[j], g);
@@ -155,8 +239,12 @@ struct Master {
 
     // Overwrite the whole state (used by tests that start both precisions from one state).
     void set_state(const double* th, const double* vv, const double* mm, const double* sv,
-                   const int64_t* it, int64_t kd, int64_t kc) {
+                   const int64_t* it, int64_t kd, int64_t kc, const double* vworkers) {
         for (int64_t j = 0; j < d; ++j) { theta[j] = (T)th[j]; v[j] = (T)vv[j]; m[j] = (T)mm[j]; }
+        if (is_dana()) {      // vv carries sum_j v^j, vworkers the N rows
+            for (int64_t j = 0; j < d; ++j) vsum[j] = (T)vv[j];
+            for (size_t q = 0; q < (size_t)n_workers * d; ++q) vw[q] = (T)vworkers[q];
+        }
         for (size_t q = 0; q < (size_t)n_workers * d; ++q) saved[q] = (T)sv[q];
         for (int i = 0; i < n_workers; ++i) iter[i] = it[i];
         k_done = kd;
@@ -197,6 +285,10 @@ Master<T>* make(int64_t d, int n, double lr, double momentum, double beta, int v
     M->m.assign(d, 0);
     M->saved.assign((size_t)n * d, 0);
     M->iter.assign(n, 0);
+    if (M->is_dana()) {
+        M->vw.assign((size_t)n * d, 0);
+        M->vsum.assign(d, 0);
+    }
     return M;
 }
 
@@ -209,7 +301,7 @@ extern "C" {
 void* gao_create(int64_t d, int n_workers, double lr, double momentum, double beta, int variant,
                  int precision) {
     if (d <= 0 || n_workers <= 0 || (precision != 32 && precision != 64)) return nullptr;
-    if (variant < 0 || variant > 2) return nullptr;
+    if (variant < 0 || variant > 6) return nullptr;
     auto* h = new (std::nothrow) Handle{precision, nullptr, nullptr};
     if (!h) return nullptr;
     try {
@@ -248,9 +340,13 @@ int64_t gao_k_done(void* p) { auto* h = (Handle*)p; return h->precision == 32 ? 
 int64_t gao_iter(void* p, int worker) { auto* h = (Handle*)p; return h->precision == 32 ? h->f->iter[worker] : h->g->iter[worker]; }
 
 void gao_set_state(void* p, const double* th, const double* v, const double* m, const double* saved,
-                   const int64_t* iter, int64_t k_done, int64_t k_c) {
+                   const int64_t* iter, int64_t k_done, int64_t k_c, const double* v_workers) {
     auto* h = (Handle*)p;
-    DISPATCH(h, set_state(th, v, m, saved, iter, k_done, k_c));
+    DISPATCH(h, set_state(th, v, m, saved, iter, k_done, k_c, v_workers));
+}
+void gao_set_dana_sum(void* p, int mode) {
+    auto* h = (Handle*)p;
+    if (h->precision == 32) h->f->dana_sum = mode; else h->g->dana_sum = mode;
 }
 int64_t gao_k_c(void* p) { auto* h = (Handle*)p; return h->precision == 32 ? h->f->k_c : h->g->k_c; }
 
@@ -260,12 +356,16 @@ void gao_stats(void* p, double* sum_gap, double* max_gap) {
     *max_gap = h->precision == 32 ? h->f->last_max_gap : h->g->last_max_gap;
 }
 
-// which: 0 theta, 1 v, 2 m, 3 C (derived from m), 4+i saved copy of worker i. Output in double.
+// which: 0 theta, 1 v (DANA: sum_j v^j), 2 m, 3 C (derived from m), 4+i saved copy of worker i,
+// 100000+i worker i's momentum v^i (DANA). Output in double.
 int gao_get(void* p, int which, double* out) {
     auto* h = (Handle*)p;
     auto copy = [&](auto* M) -> int {
         const int64_t d = M->d;
         if (which == 0) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->theta[j];
+        else if (which == 1 && M->is_dana()) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->vsum[j];
+        else if (which >= 100000 && which < 100000 + M->n_workers && M->is_dana())
+            for (int64_t j = 0; j < d; ++j) out[j] = (double)M->vw[(size_t)(which - 100000) * d + j];
         else if (which == 1) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->v[j];
         else if (which == 2) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->m[j];
         else if (which == 3) {

@@ -11,7 +11,7 @@ from fractions import Fraction
 
 import numpy as np
 
-ASGD, SA, GA = 0, 1, 2
+ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA = range(7)
 THETA, V, M, C = 0, 1, 2, 3
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
@@ -380,6 +380,232 @@ def pin_exact_brute_force(make):
                         (variant, c_order, prec, which, got, want)
 
 
+# ------------------------------------------------------------------ SA-Gradient and DANA
+def pin_sa_gradient_two_step(make):
+    """Algorithm 'Staleness-Aware-Gradient: master': v <- gamma v + g/tau, theta <- theta - eta v.
+    Unrolled twice: theta_{k+2} = theta_{k+1} - eta (gamma^2 v_k + gamma g_k/tau_k + g_{k+1}/tau_{k+1}),
+    which differs from the Section 4.1 form where the whole step is divided by tau_{k+1}."""
+    d, eta, gam = 13, 0.1, 0.9
+    r = _rng(21)
+    th0 = _f32(r.normal(size=d))
+    sched, want_tau = [0, 1, 2, 0, 2], [1, 2, 3, 3, 2]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    o = make(d, 3, eta, gam, 0.999, SA_GRAD, precision=64)
+    o.set_params(th0)
+    th, v, taus = [o.get(THETA)], [o.get(V)], []
+    for i, g in zip(sched, grads):
+        taus.append(o.push(i, g))
+        o.pull(i)
+        th.append(o.get(THETA))
+        v.append(o.get(V))
+    assert taus == want_tau
+    e, g_ = float(np.float32(eta)), float(np.float32(gam))
+    G = [g.astype(np.float64) for g in grads]
+    for k in range(len(sched) - 1):
+        two = th[k + 1] - e * (g_ * g_ * v[k] + g_ * G[k] / want_tau[k] + G[k + 1] / want_tau[k + 1])
+        assert np.allclose(th[k + 2], two, rtol=1e-13, atol=1e-14)
+    # all delays 1 (one worker): the same as plain momentum, bit for bit
+    a = make(d, 1, eta, gam, 0.999, SA_GRAD, precision=32)
+    b = make(d, 1, eta, gam, 0.999, ASGD, precision=32)
+    for o_ in (a, b):
+        o_.set_params(th0)
+        for g in grads:
+            assert o_.push(0, g) == 1
+            o_.pull(0)
+    assert np.array_equal(a.get(THETA), b.get(THETA))
+
+
+def pin_dana_one_worker_is_nesterov(make):
+    """Algorithm 'DANA: master' with one worker: the worker is always sent theta - eta gamma v,
+    the look-ahead point of Nesterov's accelerated gradient. On a quadratic the points sent are
+    exactly the iterates of torch.optim.SGD(nesterov=True), which stores that look-ahead point."""
+    import torch
+    d, eta, gam, steps = 19, 0.05, 0.9, 30
+    r = _rng(22)
+    th0 = _f32(r.normal(size=d))
+    a = r.uniform(0.5, 2.0, size=d)
+    target = r.normal(size=d)
+    p = torch.tensor(th0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([p], lr=float(np.float32(eta)), momentum=float(np.float32(gam)), nesterov=True)
+    o = make(d, 1, eta, gam, 0.999, DANA, precision=64)
+    o.set_params(th0)
+    for _ in range(steps):
+        sent = o.saved(0)
+        assert np.allclose(sent, p.detach().numpy(), rtol=1e-11, atol=1e-12)
+        g = _f32(a * (sent - target))            # gradient at the point the worker was sent
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        assert o.push(0, g) == 1
+        o.pull(0)
+    assert np.allclose(o.saved(0), p.detach().numpy(), rtol=1e-10, atol=1e-11)
+    assert not np.allclose(o.saved(0), o.get(THETA), rtol=1e-3, atol=1e-6), "the estimate is not theta itself"
+
+
+def pin_dana_zero_momentum_reduces(make):
+    """gamma = 0: the estimate is theta itself and every DANA master is its plain counterpart
+    (DANA = ASGD, DANA-SA = SA-Gradient, DANA-GA = GA), bit for bit."""
+    d, n, eta = 23, 3, 0.1
+    r = _rng(23)
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 2, 1, 0, 2, 2, 0]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    for dana, plain in ((DANA, ASGD), (DANA_SA, SA_GRAD), (DANA_GA, GA)):
+        a = make(d, n, eta, 0.0, 0.999, dana, precision=32)
+        b = make(d, n, eta, 0.0, 0.999, plain, precision=32)
+        a.set_params(th0)
+        b.set_params(th0)
+        assert a.push_batch(sched, grads) == b.push_batch(sched, grads)
+        assert np.array_equal(a.get(THETA), b.get(THETA)), (dana, plain)
+        for i in range(n):
+            assert np.array_equal(a.saved(i), b.saved(i))
+        if dana == DANA_GA:
+            assert np.array_equal(a.get(M), b.get(M)) and a.stats() == b.stats()
+
+
+def pin_dana_structure(make):
+    """DANA masters, step by step: only the arriving worker's momentum changes, v^i <- gamma v^i
+    + g (DANA) or g/tau (DANA-SA); the master moves by -eta v^i; the running sum equals the sum
+    of the N momentum vectors; the worker is sent theta - eta gamma sum_j v^j; summing the v^j
+    afresh at every send (the printed form) gives the same trajectory."""
+    d, n, eta, gam = 11, 4, 0.1, 0.9
+    r = _rng(24)
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 2, 3, 1, 0, 3, 3, 2, 1]
+    want_tau = [1, 2, 3, 4, 3, 5, 3, 1, 6, 5]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    e, g_ = float(np.float32(eta)), float(np.float32(gam))
+    for variant in (DANA, DANA_SA):
+        o = make(d, n, eta, gam, 0.999, variant, precision=64)
+        o.set_params(th0)
+        vw = [np.zeros(d) for _ in range(n)]
+        th = th0.astype(np.float64)
+        for i, g, tau in zip(sched, grads, want_tau):
+            assert o.push(i, g) == tau
+            gg = g.astype(np.float64) / (tau if variant == DANA_SA else 1)
+            vw[i] = g_ * vw[i] + gg
+            th = th - e * vw[i]
+            for w in range(n):
+                assert np.allclose(o.worker_momentum(w), vw[w], rtol=1e-13, atol=1e-15)
+            assert np.allclose(o.get(THETA), th, rtol=1e-13, atol=1e-14)
+            assert np.allclose(o.get(V), sum(vw), rtol=1e-12, atol=1e-14)
+            o.pull(i)
+            assert np.allclose(o.saved(i), th - e * g_ * sum(vw), rtol=1e-12, atol=1e-14)
+    # constant gradient, round robin: worker's momentum after t pushes is c (1-gam^t)/(1-gam)
+    c = _f32(r.normal(size=d))
+    o = make(d, 3, eta, gam, 0.999, DANA, precision=64)
+    o.set_params(th0)
+    o.push_batch([k % 3 for k in range(9)], [c] * 9)
+    geo = [(1 - g_ ** t) / (1 - g_) for t in (1, 2, 3)]
+    assert np.allclose(o.worker_momentum(1), c.astype(np.float64) * geo[2], rtol=1e-13)
+    assert np.allclose(o.get(THETA), th0.astype(np.float64) - e * 3 * sum(geo) * c.astype(np.float64), rtol=1e-12, atol=1e-13)
+    # running sum versus the printed sum over j
+    for variant in (DANA, DANA_SA, DANA_GA):
+        a = make(d, n, eta, gam, 0.999, variant, precision=64, dana_sum=1)
+        b = make(d, n, eta, gam, 0.999, variant, precision=64, dana_sum=0)
+        a.set_params(th0)
+        b.set_params(th0)
+        assert a.push_batch(sched, grads) == b.push_batch(sched, grads) == want_tau
+        assert np.allclose(a.get(THETA), b.get(THETA), rtol=1e-12, atol=1e-13)
+        for i in range(n):
+            assert np.allclose(a.saved(i), b.saved(i), rtol=1e-12, atol=1e-13)
+
+
+def pin_dana_gap(make):
+    """Algorithm 'DANA-Gap-Aware: master': the Gap is measured against the ESTIMATE that was
+    saved when sent; where the master happens to sit on that estimate the gradient passes
+    unpenalised; elsewhere it is divided by |theta - theta^i|/C + 1 with the same C as GA."""
+    d, eta, gam = 10, 0.1, 0.5
+    r = _rng(25)
+    th0 = _f32(r.normal(size=d))
+    g0 = _f32(r.normal(size=d))
+    o = make(d, 2, eta, gam, 0.75, DANA_GA, precision=64)
+    o.set_params(th0)
+    assert o.push(0, g0) == 1            # G = 1 (copy = theta_0 = master); v^0 = g0
+    assert np.array_equal(o.worker_momentum(0), g0.astype(np.float64))
+    o.pull(0)
+    e, g_ = float(np.float32(eta)), float(np.float32(gam))
+    th1 = th0.astype(np.float64) - e * g0.astype(np.float64)
+    est = th1 - e * g_ * g0.astype(np.float64)
+    assert np.allclose(o.saved(0), est, rtol=1e-14)
+    # Gap of worker 0 now: |theta_1 - estimate| / C + 1 with C = eta (|v| + eps) after one refresh
+    Cw = e * (np.abs(g0.astype(np.float64)) + 1e-8)
+    assert np.allclose(o.get(C), Cw, rtol=1e-12)
+    assert np.allclose(o.gap(0), np.abs(th1 - est) / Cw + 1, rtol=1e-12)
+    assert np.allclose(o.gap(0), g_ + 1, rtol=1e-6)       # eta gamma |v| / (eta |v|) + 1
+    # worker 1 still holds theta_0: its Gap is |theta_1 - theta_0| / C + 1 = 2
+    assert np.allclose(o.gap(1), 2.0, rtol=1e-6)
+    g1 = _f32(r.normal(size=d))
+    G1 = o.gap(1)
+    assert o.push(1, g1) == 2
+    assert np.allclose(o.worker_momentum(1), g1.astype(np.float64) / G1, rtol=1e-13)
+    assert np.allclose(o.get(THETA), th1 - e * g1.astype(np.float64) / G1, rtol=1e-13)
+
+
+def brute_force_dana(th0, sched, grads, n, eta, gam, beta, eps, variant, c_order):
+    """The three DANA masters in exact rational arithmetic; the sum over workers is the printed one."""
+    d = len(th0)
+    th = [Fraction(float(x)) for x in th0]
+    vw = [[Fraction(0)] * d for _ in range(n)]
+    m = [Fraction(0)] * d
+    saved = [list(th) for _ in range(n)]
+    it = [0] * n
+    refreshes = 0
+    taus = []
+    for k, (i, g) in enumerate(zip(sched, grads), start=1):
+        g = [Fraction(float(x)) for x in g]
+        tau = k - it[i]
+        taus.append(tau)
+        for j in range(d):
+            gp = g[j]
+            if variant == DANA_SA:
+                gp = g[j] / tau
+            elif variant == DANA_GA:
+                r, mj = refreshes, m[j]
+                if c_order == 1:
+                    u = gam * vw[i][j] + g[j]
+                    mj = beta * mj + (1 - beta) * u * u
+                    r += 1
+                    m[j] = mj
+                Cj = eta * eps if r == 0 else eta * (_sqrt_fraction(mj / (1 - beta ** r)) + eps)
+                gp = g[j] / (abs(th[j] - saved[i][j]) / Cj + 1)
+            vw[i][j] = gam * vw[i][j] + gp
+            th[j] = th[j] - eta * vw[i][j]
+            if variant == DANA_GA and c_order == 0:
+                m[j] = beta * m[j] + (1 - beta) * vw[i][j] * vw[i][j]
+        if variant == DANA_GA:
+            refreshes += 1
+        saved[i] = [th[j] - eta * gam * sum(vw[w][j] for w in range(n)) for j in range(d)]
+        it[i] = k
+    return th, vw, m, saved, taus
+
+
+def pin_dana_exact_brute_force(make):
+    """Algorithms 'DANA', 'DANA-Staleness-Aware', 'DANA-Gap-Aware: master' in exact arithmetic."""
+    r = _rng(26)
+    d, n = 3, 3
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 0, 2, 1, 0, 2]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    eta, gam, beta, eps = 0.125, 0.75, 0.875, 1e-8
+    F = Fraction
+    for variant in (DANA, DANA_SA, DANA_GA):
+        for c_order in ((0, 1) if variant == DANA_GA else (0,)):
+            th, vw, m, saved, taus = brute_force_dana(th0, sched, grads, n, F(eta), F(gam), F(beta), F(eps),
+                                                      variant, c_order)
+            for prec, tol in ((64, 2e-13), (32, 2e-5)):
+                for dana_sum in (0, 1):
+                    o = make(d, n, eta, gam, beta, variant, precision=prec, c_order=c_order, eps=eps,
+                             dana_sum=dana_sum)
+                    o.set_params(th0)
+                    assert o.push_batch(sched, grads) == taus
+                    pairs = [(o.get(THETA), th), (o.get(M), m)]
+                    pairs += [(o.worker_momentum(w), vw[w]) for w in range(n)]
+                    pairs += [(o.saved(w), saved[w]) for w in range(n)]
+                    for got, ref in pairs:
+                        want = np.array([float(x) for x in ref])
+                        assert np.all(np.abs(got - want) <= tol * (1 + np.abs(want))), (variant, c_order, prec)
+
+
 ALL_PINS = [
     pin_gap_is_one_where_copy_equals_master,
     pin_one_worker_is_heavy_ball,
@@ -392,4 +618,10 @@ ALL_PINS = [
     pin_pull_saves_master,
     pin_hand_worked_example,
     pin_exact_brute_force,
+    pin_sa_gradient_two_step,
+    pin_dana_one_worker_is_nesterov,
+    pin_dana_zero_momentum_reduces,
+    pin_dana_structure,
+    pin_dana_gap,
+    pin_dana_exact_brute_force,
 ]

@@ -55,6 +55,30 @@ MUTANTS = [
     ("adam_order_uses_penalised_v", "const T u = std::fma(gamma, v[j], (T)grad[j]);",
      "const T u = v[j];"),
     ("set_params_keeps_momentum", "v[j] = 0;\n            m[j] = 0;", "m[j] = 0;"),
+    # SA-Gradient and the DANA masters
+    ("sa_grad_multiplies", "const T g_tau = (T)grad[j] / (T)tau;", "const T g_tau = (T)grad[j] * (T)tau;"),
+    ("sa_grad_ignores_tau", "const T g_tau = (T)grad[j] / (T)tau;", "const T g_tau = (T)grad[j];"),
+    ("dana_estimate_sign", "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);",
+     "saved[(size_t)i * d + j] = std::fma(eta_gamma, total, theta[j]);"),
+    ("dana_estimate_without_gamma", "const T eta_gamma = eta * gamma;", "const T eta_gamma = eta;"),
+    ("dana_estimate_own_momentum_only", "T total = vsum[j];", "T total = vw[(size_t)i * d + j];"),
+    ("dana_sends_theta", "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);",
+     "saved[(size_t)i * d + j] = theta[j];"),
+    ("dana_shared_momentum", "T* vi = &vw[(size_t)i * d];", "T* vi = &vw[0];"),
+    ("dana_sa_ignores_tau", "g_pen = g / (T)tau;                        // DANA-SA: g / tau", "g_pen = g;"),
+    ("dana_master_uses_sum", "theta[j] = std::fma(-eta, v_new, theta[j]);    // master's weights",
+     "theta[j] = std::fma(-eta, vsum[j], theta[j]);"),
+    ("dana_sum_forgets_old", "vsum[j] = (vsum[j] - v_old) + v_new;", "vsum[j] = vsum[j] + v_new;"),
+    ("dana_momentum_dampened", "const T v_new = std::fma(gamma, v_old, g_pen);",
+     "const T v_new = std::fma(gamma, v_old, ((T)1 - gamma) * g_pen);"),
+    ("dana_gap_against_theta0", "const T dist = std::fabs(theta[j] - s[j]); // s = the estimate saved when sent",
+     "const T dist = std::fabs(theta[j] - theta[j]);"),
+    ("dana_gap_without_one", "const T G = dist / C + (T)1;\n                const T inv_gap = (T)1 / G;\n                g_pen",
+     "const T G = dist / C;\n                const T inv_gap = (T)1 / G;\n                g_pen"),
+    ("dana_ga_m_from_sum", "m[j] = std::fma(beta, m[j], one_minus_beta * (vi[j] * vi[j]));",
+     "m[j] = std::fma(beta, m[j], one_minus_beta * (vsum[j] * vsum[j]));"),
+    ("dana_pull_forgets_iteration", "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);\n        }\n        iter[i] = k_done;",
+     "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);\n        }"),
 ]
 
 
