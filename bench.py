@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--config", default="C5")
     ap.add_argument("--params", type=int, default=0, help="profiling aid: a one-segment vector of this size")
     ap.add_argument("--workers", type=int, default=32)
-    ap.add_argument("--variant", default="GA", choices=["GA", "SA", "ASGD"])
+    ap.add_argument("--variant", default="GA", choices=["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA"])
     ap.add_argument("--window", type=int, default=16)
     ap.add_argument("--math", default="exact", choices=["exact", "fast"])
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -58,9 +58,11 @@ def parse_args():
 def bytes_per_param_window(variant, k):
     """Algorithmic bytes one parameter moves in a k-arrival window (fp32): theta, v (and m) in
     and out once; per arrival the gradient (and, for GA, the saved copy) in and the saved copy out."""
-    if variant == "GA":
-        return 24 + 12 * k
-    return 16 + 8 * k
+    state = 24 if variant in ("GA", "DANA_GA") else 16          # theta, v or sum_j v^j (, m) in and out
+    per_arrival = 8 + (4 if variant in ("GA", "DANA_GA") else 0)  # gradient in, sent copy out (, saved copy in)
+    if variant.startswith("DANA"):
+        per_arrival += 8                                           # the worker's v^i in and out
+    return state + per_arrival * k
 
 
 def hbm_peak():
@@ -155,7 +157,7 @@ def time_oracle(wl, variant, n_params, windows_list, seed_offset=0):
     j0 = min(j0, wl.d - n_params)
     idx = np.arange(j0, j0 + n_params, dtype=np.int64)
     o = oracle.Oracle(n_params, wl.n_workers, wl.lr, wl.momentum, wl.c_beta,
-                      {"ASGD": oracle.ASGD, "SA": oracle.SA, "GA": oracle.GA}[variant], precision=32)
+                      oracle.VARIANTS[variant], precision=32)
     o.set_params(wl.theta0(idx))
     k, updates, seconds = 0, 0, 0.0
     for win in windows_list:

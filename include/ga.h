@@ -40,12 +40,21 @@ typedef struct ga_engine ga_engine;
 enum {
     GA_ASGD = 0, /* Algorithm "Momentum-ASGD: master" (Section 4)                      */
     GA_SA = 1,   /* Algorithm "Staleness-Aware: master" (Section 4.1): step eta / tau   */
-    GA_GA = 2    /* Algorithm "Gap-Aware: master" (Section 5), parameter-wise Gap (5.3) */
+    GA_GA = 2,   /* Algorithm "Gap-Aware: master" (Section 5), parameter-wise Gap (5.3) */
+    GA_SA_GRAD = 3, /* Algorithm "Staleness-Aware-Gradient: master" (appendix): gradient / tau */
+    /* The DANA masters (appendix, Algorithms "DANA: master", "DANA-Staleness-Aware: master",
+     * "DANA-Gap-Aware: master"): one momentum vector v^i per worker; the master moves by
+     * -eta v^i; a pull sends (and saves) the look-ahead estimate theta - eta gamma sum_j v^j.
+     * The sum is kept as a running sum, (sum - old v^i) + new v^i. Costs one more N x n_params
+     * array of device memory. */
+    GA_DANA = 4,    /* v^i <- gamma v^i + g                                   */
+    GA_DANA_SA = 5, /* v^i <- gamma v^i + g / tau                             */
+    GA_DANA_GA = 6  /* v^i <- gamma v^i + (1/G) g, Gap against the saved estimate */
 };
 
 enum { GA_OK = 0, GA_ERR_ARG = -1, GA_ERR_STATE = -2, GA_ERR_OOM = -3, GA_ERR_CUDA = -4 };
 
-/* vectors readable with ga_get */
+/* vectors readable with ga_get; GA_V is the master's momentum v, or sum_j v^j for the DANA variants */
 enum { GA_THETA = 0, GA_V = 1, GA_M = 2, GA_C = 3 };
 
 /* options for ga_set_option */
@@ -86,7 +95,8 @@ int ga_set_stream(ga_engine* e, void* cuda_stream);
 int ga_set_params(ga_engine* e, const float* theta0_dev);
 
 /* "Send theta to worker i" (Algorithm "Momentum-ASGD: worker": "Receive parameters"): copies the
- * master parameters into worker's saved copy with TMA bulk copies, records iter[worker] <-
+ * master parameters into worker's saved copy with TMA bulk copies (the DANA variants compute and
+ * store the estimate theta - eta gamma sum_j v^j instead), records iter[worker] <-
  * arrivals applied so far, and returns the device address of that copy (library-owned, stable for
  * the engine's life; contents change at that worker's next pull or batched push). NULL on error. */
 const float* ga_pull(ga_engine* e, int worker);
@@ -128,6 +138,10 @@ int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* cons
  * stands (GA_C; last two lines of the C algorithm) into out_dev (n_params floats). */
 int ga_get(ga_engine* e, int which, float* out_dev);
 
+/* DANA variants only: copy worker's momentum vector v^worker into out_dev (n_params floats).
+ * GA_ERR_STATE for the other variants. */
+int ga_get_worker_momentum(ga_engine* e, int worker, float* out_dev);
+
 /* The parameter-wise Gap |theta - theta^worker| / C + 1 (Section 5.3) of `worker` against the
  * master as it stands, into gap_out_dev (n_params floats). Changes no state. */
 int ga_gap(ga_engine* e, int worker, float* gap_out_dev);
@@ -143,9 +157,9 @@ int64_t ga_num_arrivals(ga_engine* e);
 int64_t ga_worker_iter(ga_engine* e, int worker);
 
 /* Checkpoint: all state needed to continue bit-identically (hyper-parameters, options, counters,
- * iter[], theta, v, m, saved copies). ga_export_state returns the number of bytes needed; it
+ * iter[], theta, v, m, saved copies, and the workers' momentum vectors for DANA). ga_export_state returns the number of bytes needed; it
  * writes them when cap is large enough (buf_host may be NULL to query). ga_import_state needs an
- * engine created with the same n_params and n_workers. */
+ * engine created with the same n_params, n_workers and variant. */
 size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap);
 int ga_import_state(ga_engine* e, const void* buf_host, size_t len);
 

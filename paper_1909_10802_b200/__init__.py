@@ -15,13 +15,14 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("GA_LIBRARY") or os.path.join(_HERE, "libga.so")   # GA_LIBRARY: another build
 
-GA_ASGD, GA_SA, GA_GA = 0, 1, 2
+GA_ASGD, GA_SA, GA_GA, GA_SA_GRAD, GA_DANA, GA_DANA_SA, GA_DANA_GA = range(7)
 GA_OK, GA_ERR_ARG, GA_ERR_STATE, GA_ERR_OOM, GA_ERR_CUDA = 0, -1, -2, -3, -4
 GA_THETA, GA_V, GA_M, GA_C = 0, 1, 2, 3
 GA_OPT_C_ORDER, GA_OPT_MATH, GA_OPT_STATS, GA_OPT_WINDOW = 0, 1, 2, 3
 GA_MAX_WINDOW = 16
 GA_NOALLOC_MAX_PARAMS = 1 << 28
-VARIANTS = {"ASGD": GA_ASGD, "SA": GA_SA, "GA": GA_GA}
+VARIANTS = {"ASGD": GA_ASGD, "SA": GA_SA, "GA": GA_GA, "SA_GRAD": GA_SA_GRAD, "DANA": GA_DANA,
+            "DANA_SA": GA_DANA_SA, "DANA_GA": GA_DANA_GA}
 
 # every symbol include/ga.h declares: name -> (restype, argtypes)
 _c = ctypes
@@ -36,6 +37,7 @@ _SIGNATURES = {
     "ga_push_batch": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p]),
     "ga_push_batch_host": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
     "ga_get": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p]),
+    "ga_get_worker_momentum": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p]),
     "ga_gap": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p]),
     "ga_set_option": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_double]),
     "ga_get_stats": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
@@ -210,6 +212,13 @@ class Engine:
         _check(self._l.ga_get(self._h, which, _ptr(out)))
         return out
 
+    def get_worker_momentum(self, worker, out=None):
+        torch = self._torch
+        if out is None:
+            out = torch.empty(self.n_params, dtype=torch.float32, device="cuda")
+        _check(self._l.ga_get_worker_momentum(self._h, worker, _ptr(out)))
+        return out
+
     def gap(self, worker, out=None):
         torch = self._torch
         if out is None:
@@ -260,10 +269,13 @@ def unpack_state(blob):
     off = hs
     iters = np.frombuffer(blob, dtype=np.int64, count=n, offset=off).copy()
     off += 8 * n
-    vecs = np.frombuffer(blob, dtype=np.float32, count=(3 + n) * d, offset=off).reshape(3 + n, d).copy()
-    return dict(d=d, n_workers=n, k_done=k_done, k_c=k_c, lr=lr, momentum=gamma, c_beta=beta, eps=eps,
+    dana = variant in (GA_DANA, GA_DANA_SA, GA_DANA_GA)
+    rows = 3 + n * (2 if dana else 1)
+    vecs = np.frombuffer(blob, dtype=np.float32, count=rows * d, offset=off).reshape(rows, d).copy()
+    extra = {"v_workers": vecs[3 + n:]} if dana else {}
+    return dict(**extra, d=d, n_workers=n, k_done=k_done, k_c=k_c, lr=lr, momentum=gamma, c_beta=beta, eps=eps,
                 variant=variant, c_order=c_order, fast_math=fast_math, stats=stats, window=window,
-                iter=iters, theta=vecs[0], v=vecs[1], m=vecs[2], saved=vecs[3:])
+                iter=iters, theta=vecs[0], v=vecs[1], m=vecs[2], saved=vecs[3:3 + n])
 
 
 def pack_state(st):
@@ -275,7 +287,7 @@ def pack_state(st):
                        st["momentum"], st["c_beta"], st["eps"], st["variant"], st["c_order"],
                        st["fast_math"], st["stats"], st["window"], 0)
     parts = [head, np.ascontiguousarray(st["iter"], dtype=np.int64).tobytes()]
-    for name in ("theta", "v", "m", "saved"):
+    for name in ("theta", "v", "m", "saved") + (("v_workers",) if "v_workers" in st else ()):
         a = np.ascontiguousarray(st[name], dtype=np.float32)
         parts.append(a.tobytes())
     return b"".join(parts)

@@ -40,6 +40,7 @@ struct ga_engine {
     float lr = 0, gamma = 0, beta = 0, eps = 1e-8f;
     int c_order = 0, fast_math = 0, stats = 0, window = GA_MAX_WINDOW;
     float *theta = nullptr, *vel = nullptr, *mom = nullptr, *saved = nullptr;
+    float* vworker = nullptr;     // DANA: N rows, v^i of every worker (vel then holds their sum)
     std::vector<int64_t> iter;
     int64_t k_done = 0, k_c = 0;
     cudaStream_t stream = nullptr;
@@ -59,6 +60,10 @@ struct ga_engine {
     cudaEvent_t ev_h2d[2] = {nullptr, nullptr}, ev_kernel[2] = {nullptr, nullptr}, ev_prev = nullptr;
 
     float* row(int i) const { return saved + (size_t)i * stride; }
+    float* vrow(int i) const { return vworker ? vworker + (size_t)i * stride : nullptr; }
+    bool is_dana() const { return variant == GA_DANA || variant == GA_DANA_SA || variant == GA_DANA_GA; }
+    bool is_gap() const { return variant == GA_GA || variant == GA_DANA_GA; }
+    bool is_tau_grad() const { return variant == GA_SA_GRAD || variant == GA_DANA_SA; }
     ga::Hyper hyper() const {
         ga::Hyper h;
         h.eta_max = lr;
@@ -66,6 +71,7 @@ struct ga_engine {
         h.beta = beta;
         h.one_minus_beta = (float)(1.0 - (double)beta);
         h.eps = eps;
+        h.eta_gamma = lr * gamma;
         return h;
     }
     // 1/(1-beta^k) for the C in force after k refreshes of m; 0 before the first (C = eta_max*eps)
@@ -133,32 +139,28 @@ int grid_1d(long long n, int threads, int cap) {
 }
 
 // ----------------------------------------------------------------------------- launch
-template <int VARIANT, bool EXACT, int C_ORDER, bool STATS>
+template <int FAMILY, int PENALTY, bool EXACT, int C_ORDER, bool STATS>
 void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st) {
     const long long nvec = vec_end - vec_begin;
     long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
     // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner
     if (w.K == 1)
-        ga::ga_window_kernel<VARIANT, EXACT, C_ORDER, STATS, 1><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
+        ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, 1><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
             e->theta, e->vel, e->mom, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
     else
-        ga::ga_window_kernel<VARIANT, EXACT, C_ORDER, STATS, GA_WINDOW_BATCH><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
+        ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, GA_WINDOW_BATCH><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
             e->theta, e->vel, e->mom, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
     if (STATS) {
         ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev);
     }
 }
 
-int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st,
-                  bool allow_stats = true) {
-    if (vec_end <= vec_begin || w.K <= 0) return GA_OK;
-    const bool exact = !e->fast_math;
-    const bool stats = allow_stats && e->stats && e->variant == GA_GA;
-    if (e->variant == GA_ASGD) launch_window_t<ga::ASGD, true, 0, false>(e, w, vec_begin, vec_end, st);
-    else if (e->variant == GA_SA) launch_window_t<ga::SA, true, 0, false>(e, w, vec_begin, vec_end, st);
-    else {
-#define GA_CASE(EX, CO, ST) launch_window_t<ga::GA, EX, CO, ST>(e, w, vec_begin, vec_end, st)
+template <int FAMILY>
+void launch_family(ga_engine* e, const ga::Window& w, long long vb, long long ve, cudaStream_t st, bool stats) {
+    if (e->is_gap()) {
+        const bool exact = !e->fast_math;
+#define GA_CASE(EX, CO, ST) launch_window_t<FAMILY, ga::PEN_GAP, EX, CO, ST>(e, w, vb, ve, st)
         if (exact) {
             if (e->c_order == 0) { if (stats) GA_CASE(true, 0, true); else GA_CASE(true, 0, false); }
             else { if (stats) GA_CASE(true, 1, true); else GA_CASE(true, 1, false); }
@@ -167,7 +169,19 @@ int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long l
             else { if (stats) GA_CASE(false, 1, true); else GA_CASE(false, 1, false); }
         }
 #undef GA_CASE
+    } else if (e->is_tau_grad()) {
+        launch_window_t<FAMILY, ga::PEN_TAU, true, 0, false>(e, w, vb, ve, st);
+    } else {
+        launch_window_t<FAMILY, ga::PEN_NONE, true, 0, false>(e, w, vb, ve, st);
     }
+}
+
+int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st,
+                  bool allow_stats = true) {
+    if (vec_end <= vec_begin || w.K <= 0) return GA_OK;
+    const bool stats = allow_stats && e->stats && e->is_gap();
+    if (e->is_dana()) launch_family<ga::DANA>(e, w, vec_begin, vec_end, st, stats);
+    else launch_family<ga::MOM>(e, w, vec_begin, vec_end, st, stats);
     GA_CUDA(e, cudaGetLastError());
     if (stats) { e->stats_valid = true; e->stats_slot = w.K - 1; }
     return GA_OK;
@@ -186,8 +200,10 @@ void fill_window(ga_engine* e, ga::Window& w, const int* workers, const float* c
         if (delays) delays[j] = tau;
         w.grad[j] = grads[j];
         w.saved[j] = e->row(i);
+        w.vworker[j] = e->vrow(i);
+        w.tau[j] = (float)tau;
         w.eta_eff[j] = e->variant == GA_SA ? e->lr / (float)tau : e->lr;
-        if (e->variant == GA_GA) {
+        if (e->is_gap()) {
             // the C in force for this arrival: after k_c refreshes (lagged order), or after
             // this arrival's own refresh (Adam order)
             w.inv_bias[j] = e->inv_bias(e->c_order == 0 ? e->k_c : e->k_c + 1);
@@ -201,6 +217,8 @@ void fill_window(ga_engine* e, ga::Window& w, const int* workers, const float* c
     for (int j = K; j < ga::kMaxWindow; ++j) {
         w.grad[j] = nullptr;
         w.saved[j] = nullptr;
+        w.vworker[j] = nullptr;
+        w.tau[j] = 1.f;
         w.inv_bias[j] = 0.f;
         w.eta_eff[j] = 0.f;
     }
@@ -262,7 +280,7 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
     if (!(lr > 0.f) || !std::isfinite(lr)) { fail(GA_ERR_ARG, "lr must be positive and finite"); return nullptr; }
     if (!(std::fabs(momentum) < 1.f)) { fail(GA_ERR_ARG, "|momentum| must be < 1"); return nullptr; }
     if (!(c_beta >= 0.f && c_beta < 1.f)) { fail(GA_ERR_ARG, "c_beta must be in [0, 1)"); return nullptr; }
-    if (variant != GA_ASGD && variant != GA_SA && variant != GA_GA) { fail(GA_ERR_ARG, "unknown variant %d", variant); return nullptr; }
+    if (variant < GA_ASGD || variant > GA_DANA_GA) { fail(GA_ERR_ARG, "unknown variant %d", variant); return nullptr; }
     ga_engine* e = new (std::nothrow) ga_engine();
     if (!e) { fail(GA_ERR_OOM, "out of host memory"); return nullptr; }
     e->d = (long long)n_params;
@@ -288,12 +306,14 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
               cudaMalloc(&e->saved, row_bytes * (size_t)n_workers) == cudaSuccess &&
               cudaMalloc(&e->partials, sizeof(ga::StatsPartial) * (size_t)e->stats_blocks * ga::kMaxWindow) == cudaSuccess &&
               cudaMalloc(&e->stats_dev, sizeof(double) * 2 * ga::kMaxWindow) == cudaSuccess &&
-              cudaMalloc(&e->pull_err, sizeof(int)) == cudaSuccess;
+              cudaMalloc(&e->pull_err, sizeof(int)) == cudaSuccess &&
+              (!e->is_dana() || cudaMalloc(&e->vworker, row_bytes * (size_t)n_workers) == cudaSuccess);
     if (ok) {
         ok = cudaMemset(e->theta, 0, row_bytes) == cudaSuccess && cudaMemset(e->vel, 0, row_bytes) == cudaSuccess &&
              cudaMemset(e->mom, 0, row_bytes) == cudaSuccess &&
              cudaMemset(e->saved, 0, row_bytes * (size_t)n_workers) == cudaSuccess &&
              cudaMemset(e->pull_err, 0, sizeof(int)) == cudaSuccess &&
+             (!e->vworker || cudaMemset(e->vworker, 0, row_bytes * (size_t)n_workers) == cudaSuccess) &&
              cudaFuncSetAttribute(ga::ga_pull_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   ga::kPullStages * ga::kPullChunk) == cudaSuccess &&
              cudaDeviceSynchronize() == cudaSuccess;
@@ -315,6 +335,7 @@ void ga_destroy(ga_engine* e) {
     cudaFree(e->vel);
     cudaFree(e->mom);
     cudaFree(e->saved);
+    cudaFree(e->vworker);
     cudaFree(e->partials);
     cudaFree(e->stats_dev);
     cudaFree(e->pull_err);
@@ -341,7 +362,7 @@ int ga_set_params(ga_engine* e, const float* theta0_dev) {
     if (int rc = check_dev_ptr(theta0_dev, "theta0_dev")) return rc;
     DeviceGuard guard(e->device);
     ga::ga_set_params_kernel<<<grid_1d(e->stride, 256, 148 * 8), 256, 0, e->stream>>>(
-        theta0_dev, e->theta, e->vel, e->mom, e->saved, e->n_workers, e->d, e->stride);
+        theta0_dev, e->theta, e->vel, e->mom, e->saved, e->vworker, e->n_workers, e->d, e->stride);
     GA_CUDA(e, cudaGetLastError());
     std::fill(e->iter.begin(), e->iter.end(), 0);
     e->k_done = 0;
@@ -353,6 +374,14 @@ int ga_set_params(ga_engine* e, const float* theta0_dev) {
 const float* ga_pull(ga_engine* e, int worker) {
     if (check_engine(e) || check_worker(e, worker)) return nullptr;
     DeviceGuard guard(e->device);
+    if (e->is_dana()) {   // the worker is sent the look-ahead estimate, not theta
+        ga::ga_pull_estimate_kernel<<<grid_1d(e->stride, 256, 148 * 8), 256, 0, e->stream>>>(
+            e->theta, e->vel, e->hyper().eta_gamma, e->stride, e->row(worker));
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) { cuda_fail(e, err, "ga_pull launch"); return nullptr; }
+        e->iter[worker] = e->k_done;
+        return e->row(worker);
+    }
     const long long bytes = e->stride * (long long)sizeof(float);
     const long long chunks = (bytes + ga::kPullChunk - 1) / ga::kPullChunk;
     const int grid = (int)(chunks < 148 * 3 ? chunks : 148 * 3);
@@ -474,6 +503,17 @@ int ga_get(ga_engine* e, int which, float* out_dev) {
     return check_pull_flag(e);
 }
 
+int ga_get_worker_momentum(ga_engine* e, int worker, float* out_dev) {
+    if (int rc = check_engine(e)) return rc;
+    if (int rc = check_worker(e, worker)) return rc;
+    if (int rc = check_dev_ptr(out_dev, "out_dev")) return rc;
+    if (!e->is_dana()) return fail(GA_ERR_STATE, "only the DANA variants keep a momentum vector per worker");
+    DeviceGuard guard(e->device);
+    GA_CUDA(e, cudaMemcpyAsync(out_dev, e->vrow(worker), sizeof(float) * (size_t)e->d, cudaMemcpyDeviceToDevice, e->stream));
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    return GA_OK;
+}
+
 int ga_gap(ga_engine* e, int worker, float* gap_out_dev) {
     if (int rc = check_engine(e)) return rc;
     if (int rc = check_worker(e, worker)) return rc;
@@ -548,7 +588,8 @@ struct StateHeader {
 size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
     if (check_engine(e)) return 0;
     const size_t vec = sizeof(float) * (size_t)e->d;
-    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * (3 + (size_t)e->n_workers);
+    const size_t rows = 3 + (size_t)e->n_workers * (e->is_dana() ? 2 : 1);
+    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows;
     if (!buf_host || cap < need) return need;
     DeviceGuard guard(e->device);
     StateHeader h{};
@@ -565,6 +606,8 @@ size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
         err = cudaMemcpyAsync(p, vecs[q], vec, cudaMemcpyDeviceToHost, e->stream);
     for (int i = 0; i < e->n_workers && err == cudaSuccess; ++i, p += vec)
         err = cudaMemcpyAsync(p, e->row(i), vec, cudaMemcpyDeviceToHost, e->stream);
+    for (int i = 0; e->is_dana() && i < e->n_workers && err == cudaSuccess; ++i, p += vec)
+        err = cudaMemcpyAsync(p, e->vrow(i), vec, cudaMemcpyDeviceToHost, e->stream);
     if (err == cudaSuccess) err = cudaStreamSynchronize(e->stream);
     if (err != cudaSuccess) { cuda_fail(e, err, "ga_export_state"); return 0; }
     return need;
@@ -579,9 +622,11 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
     if (h.d != e->d || h.n_workers != e->n_workers)
         return fail(GA_ERR_ARG, "state is for %lld parameters / %lld workers", (long long)h.d, (long long)h.n_workers);
     const size_t vec = sizeof(float) * (size_t)e->d;
-    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * (3 + (size_t)e->n_workers);
+    if (h.variant != e->variant) return fail(GA_ERR_ARG, "state is for variant %d, engine is variant %d", h.variant, e->variant);
+    const size_t rows = 3 + (size_t)e->n_workers * (e->is_dana() ? 2 : 1);
+    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows;
     if (len < need) return fail(GA_ERR_ARG, "state buffer truncated");
-    if (h.variant < GA_ASGD || h.variant > GA_GA || h.window < 1 || h.window > GA_MAX_WINDOW || h.k_done < 0 || h.k_c < 0)
+    if ( h.window < 1 || h.window > GA_MAX_WINDOW || h.k_done < 0 || h.k_c < 0)
         return fail(GA_ERR_ARG, "state header holds invalid values");
     DeviceGuard guard(e->device);
     const char* p = (const char*)buf_host + sizeof h;
@@ -592,11 +637,13 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
         GA_CUDA(e, cudaMemcpyAsync(vecs[q], p, vec, cudaMemcpyHostToDevice, e->stream));
     for (int i = 0; i < e->n_workers; ++i, p += vec)
         GA_CUDA(e, cudaMemcpyAsync(e->row(i), p, vec, cudaMemcpyHostToDevice, e->stream));
+    for (int i = 0; e->is_dana() && i < e->n_workers; ++i, p += vec)
+        GA_CUDA(e, cudaMemcpyAsync(e->vrow(i), p, vec, cudaMemcpyHostToDevice, e->stream));
     GA_CUDA(e, cudaStreamSynchronize(e->stream));
     e->iter = iter;
     e->k_done = h.k_done; e->k_c = h.k_c;
     e->lr = h.lr; e->gamma = h.gamma; e->beta = h.beta; e->eps = h.eps;
-    e->variant = h.variant; e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window;
+    e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window;
     e->stats_valid = false;
     return GA_OK;
 }
@@ -701,7 +748,7 @@ extern "C" int ga_gap_stats_noalloc(const float* theta_dev, const float* saved_d
     ga::StatsPartial* scratch = nullptr;
     if (int rc = noalloc_scratch(&scratch)) return rc;
     ga::Hyper h;
-    h.eta_max = lr_max; h.gamma = 0.f; h.beta = c_beta; h.one_minus_beta = (float)(1.0 - (double)c_beta); h.eps = 1e-8f;
+    h.eta_max = lr_max; h.gamma = 0.f; h.eta_gamma = 0.f; h.beta = c_beta; h.one_minus_beta = (float)(1.0 - (double)c_beta); h.eps = 1e-8f;
     const float inv_bias = n_refreshes == 0 ? 0.f : (float)(1.0 / (1.0 - std::pow((double)c_beta, (double)n_refreshes)));
     const int blocks = (int)((n_params + kNoAllocTile - 1) / kNoAllocTile);
     cudaStream_t st = (cudaStream_t)cuda_stream;

@@ -11,7 +11,7 @@ def run_oracle(wl, variant, n_arrivals=None, idx=None, precision=32, c_order=0, 
     (theta, v, m)} for the requested checkpoints)."""
     d = wl.d if idx is None else len(idx)
     o = oracle.Oracle(d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta,
-                      {"ASGD": oracle.ASGD, "SA": oracle.SA, "GA": oracle.GA}[variant],
+                      oracle.VARIANTS[variant],
                       precision=precision, c_order=c_order)
     o.set_params(wl.theta0(idx))
     sched = (schedule if schedule is not None else wl.schedule())

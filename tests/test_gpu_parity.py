@@ -54,12 +54,20 @@ def _compare_engine(P, run, o, idx=None, label=""):
     import torch
     sel = None if idx is None else torch.as_tensor(idx, device="cuda")
     names = (("theta", P.GA_THETA, o.THETA), ("v", P.GA_V, o.V))
-    if run.engine.variant == P.GA_GA:
+    if run.engine.variant in (P.GA_GA, P.GA_DANA_GA):
         names += (("m", P.GA_M, o.M), ("C", P.GA_C, o.C))
+    if run.engine.variant in (P.GA_DANA, P.GA_DANA_SA, P.GA_DANA_GA):
+        names += tuple((f"v^{i}", ("vw", i), None) for i in range(run.engine.n_workers))
+    names += tuple((f"sent^{i}", ("sent", i), None) for i in range(min(run.engine.n_workers, 8)))
     for name, which, owhich in names:
-        got = run.engine.get(which)
+        if isinstance(which, tuple):
+            kind, i = which
+            got = run.engine.get_worker_momentum(i) if kind == "vw" else run.engine.saved(i)
+            ref = o.worker_momentum(i) if kind == "vw" else o.saved(i)
+        else:
+            got = run.engine.get(which)
+            ref = o.get(owhich)
         got = _np(got if sel is None else got[sel])
-        ref = o.get(owhich)
         assert _close(got, ref), f"{label}{name}: outside {TOL}*(1+|ref|)"
         nbad = int(np.sum(~((got == ref.astype(np.float32)) | (np.isnan(got) & np.isnan(ref)))))
         assert nbad == 0, f"{label}{name}: {nbad} elements differ from the fp32 oracle in some bit"
@@ -97,12 +105,15 @@ def test_device_generator_sparse_rows_and_subrange(P):
 
 
 # ----------------------------------------------------------------------------- small, exhaustive
-@pytest.mark.parametrize("variant", ["GA", "SA", "ASGD"])
+ALL_VARIANTS = ["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA"]
+
+
+@pytest.mark.parametrize("variant", ALL_VARIANTS)
 @pytest.mark.parametrize("window", [1, 4, 16])
 def test_mini_trajectory(P, variant, window):
     from paper_1909_10802_b200.runner import Run
     wl = W.config("mini")
-    for c_order in ((0, 1) if variant == "GA" else (0,)):
+    for c_order in ((0, 1) if variant in ("GA", "DANA_GA") else (0,)):
         run = Run(wl, variant, window, options={P.GA_OPT_C_ORDER: c_order})
         delays = run.run()
         o, odelays, _ = run_oracle(wl, variant, c_order=c_order)
@@ -176,6 +187,52 @@ def test_c3_window_invariance(P):
                 assert all(torch.equal(a, b) for a, b in zip(ref, full)), "K=1 and K=4 disagree"
         run.close()
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("variant", ["DANA_GA", "DANA", "DANA_SA", "SA_GRAD"])
+def test_c3_dana_and_sa_gradient(P, variant):
+    """The appendix's masters on the ResNet-50 shape (64 workers), fused windows of 16."""
+    import torch
+    _sampled(P, "C3", variant, 16, n_arrivals=400).close()
+    torch.cuda.empty_cache()
+
+
+def test_dana_push_then_pull_and_checkpoint(P):
+    """DANA-GA through the stand-alone calls (the pull computes the look-ahead estimate) and
+    through export/import (the workers' momentum vectors travel with the state)."""
+    import torch
+    eng, o, rng = _small_engine(P, n=3, variant=P.GA_DANA_GA)
+    for step, i in enumerate([0, 1, 1, 2, 0]):
+        g = rng.normal(size=eng.n_params).astype(np.float32)
+        assert eng.push(i, torch.from_numpy(g).cuda()) == o.push(i, g)
+        if step != 1:
+            sent = eng.pull(i)
+            o.pull(i)
+            assert _same(_np(sent), o.saved(i))
+    blob = eng.export_state()
+    other = P.Engine(eng.n_params, 3, 0.1, 0.9, 0.999, P.GA_DANA_GA)
+    other.import_state(blob)
+    wrong = P.Engine(eng.n_params, 3, 0.1, 0.9, 0.999, P.GA_GA)
+    with pytest.raises(P.GaError):
+        wrong.import_state(blob)
+    wrong.close()
+    g = rng.normal(size=eng.n_params).astype(np.float32)
+    for e_ in (eng, other):
+        assert e_.push_batch([2], [torch.from_numpy(g).cuda()]) == [2]
+    o.push_batch([2], [g])
+    for e_ in (eng, other):
+        for which, ow in ((P.GA_THETA, o.THETA), (P.GA_V, o.V), (P.GA_M, o.M)):
+            assert _same(_np(e_.get(which)), o.get(ow))
+        for i in range(3):
+            assert _same(_np(e_.get_worker_momentum(i)), o.worker_momentum(i))
+            assert _same(_np(e_.saved(i)), o.saved(i))
+        e_.close()
+    with pytest.raises(P.GaError):
+        plain = P.Engine(100, 2)
+        try:
+            plain.get_worker_momentum(0)
+        finally:
+            plain.close()
 
 
 def test_c4_stragglers(P):
