@@ -13,9 +13,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ga_oracle.cpp")
 _LIB = os.path.join(_HERE, "libga_oracle.so")
 
-ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA = range(7)
+ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA, ADAM, ADAM_SA, ADAM_GA = range(10)
 VARIANTS = {"ASGD": ASGD, "SA": SA, "GA": GA, "SA_GRAD": SA_GRAD, "DANA": DANA, "DANA_SA": DANA_SA,
-            "DANA_GA": DANA_GA}
+            "DANA_GA": DANA_GA, "ADAM": ADAM, "ADAM_SA": ADAM_SA, "ADAM_GA": ADAM_GA}
 CXXFLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-Wall", "-Wextra"]
 
 
@@ -48,6 +48,7 @@ def _bind(path):
     lib.gao_iter.argtypes = [c.c_void_p, c.c_int]
     lib.gao_set_state.argtypes = [c.c_void_p] * 6 + [c.c_int64, c.c_int64, c.c_void_p]
     lib.gao_set_dana_sum.argtypes = [c.c_void_p, c.c_int]
+    lib.gao_set_adam.argtypes = [c.c_void_p, c.c_double, c.c_double]
     lib.gao_k_c.restype = c.c_int64
     lib.gao_k_c.argtypes = [c.c_void_p]
     lib.gao_stats.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
@@ -79,7 +80,8 @@ class Oracle:
     THETA, V, M, C = 0, 1, 2, 3
 
     def __init__(self, n_params, n_workers, lr, momentum, c_beta, variant, precision=32,
-                 c_order=0, eps=None, dana_sum=1, _lib=None):
+                 c_order=0, eps=None, dana_sum=1, beta2=0.999, adam_eps=1e-8, _lib=None):
+        """For the Adam variants `momentum` is beta_1."""
         self._l = _lib if _lib is not None else lib()
         self.d, self.n = int(n_params), int(n_workers)
         self._h = self._l.gao_create(self.d, self.n, lr, momentum, c_beta, variant, precision)
@@ -88,6 +90,7 @@ class Oracle:
         self.variant = variant
         self._l.gao_set_c_order(self._h, c_order)
         self._l.gao_set_dana_sum(self._h, dana_sum)
+        self._l.gao_set_adam(self._h, beta2, adam_eps)
         if eps is not None:
             self._l.gao_set_eps(self._h, eps)
 
@@ -132,6 +135,14 @@ class Oracle:
         """DANA: v^worker."""
         return self.get(100000 + worker)
 
+    def second_moment(self):
+        """Adam: v (the first moment is get(V))."""
+        return self.get(200000)
+
+    @property
+    def is_adam(self):
+        return self.variant in (ADAM, ADAM_SA, ADAM_GA)
+
     @property
     def is_dana(self):
         return self.variant in (DANA, DANA_SA, DANA_GA)
@@ -159,6 +170,8 @@ class Oracle:
                self.k_done, int(self._l.gao_k_c(self._h)))
         if self.is_dana:
             out += (np.stack([self.worker_momentum(i) for i in range(self.n)]),)
+        if self.is_adam:
+            out += (self.second_moment(),)
         return out
 
     def set_state(self, theta, v, m, saved, iters, k_done, k_c, v_workers=None):
@@ -169,6 +182,9 @@ class Oracle:
         if self.is_dana:
             vw = np.ascontiguousarray(v_workers, dtype=np.float64)
             assert vw.shape == (self.n, self.d)
+        if self.is_adam:      # the extra array is Adam's second moment
+            vw = np.ascontiguousarray(v_workers, dtype=np.float64)
+            assert vw.shape == (self.d,)
         self._l.gao_set_state(self._h, *(x.ctypes.data for x in a), it.ctypes.data, k_done, k_c,
                               None if vw is None else vw.ctypes.data)
 

@@ -16,6 +16,9 @@
 //   pull               : "Send theta_{k+1} to worker i" / "Save and send current
 //                        parameters" of the three master algorithms; the saved copy is
 //                        the theta^i = theta_{k-tau_k} of the appendix's remark
+//   push, ADAM*        : Algorithms "Adam: master", "Adam-Staleness-Aware: master" and
+//                        "Adam-Gap-Aware: master" (appendix): the penalty (1/tau or 1/G) enters
+//                        the first moment only
 //   momentum           : Section 3, the variant without dampening: v <- gamma v + g
 //   push, SA_GRAD      : Algorithm "Staleness-Aware-Gradient: master" (appendix): g / tau
 //   push/pull, DANA*   : Algorithms "DANA: master", "DANA-Staleness-Aware: master" and
@@ -42,6 +45,12 @@
 //     sum, S <- (S - v^i_old) + v^i_new at each arrival (what a master would do; default);
 //     0 = the printed sum_{j=1..N} v^j evaluated afresh, in order, at every send. The two are
 //     equal in exact arithmetic and are pinned against each other.
+//   * Adam-GA's C: the C algorithm needs an "update step gamma v + g", and Adam has no momentum
+//     coefficient, so it is run with gamma = 0: m is the running second moment of the raw
+//     gradient with the constant beta given at creation (its own state, separate from Adam's
+//     v); c_order decides as before whether the Gap sees m before or after this arrival's refresh.
+//   * Adam's bias corrections use k = the arrival index; m_hat = m * (1/(1-beta1^k)) with the
+//     reciprocal formed in double and rounded once, as for C.
 //   * Arithmetic: every line below is one IEEE operation per symbol, in the order
 //     written, with v <- gamma*v + g_hat and theta <- theta - eta*v each a single fused
 //     multiply-add. Build with -ffp-contract=off so nothing else is fused.
@@ -62,7 +71,8 @@
 
 namespace {
 
-enum Variant { ASGD = 0, SA = 1, GA = 2, SA_GRAD = 3, DANA = 4, DANA_SA = 5, DANA_GA = 6 };
+enum Variant { ASGD = 0, SA = 1, GA = 2, SA_GRAD = 3, DANA = 4, DANA_SA = 5, DANA_GA = 6,
+               ADAM = 7, ADAM_SA = 8, ADAM_GA = 9 };
 
 template <typename T>
 struct Master {
@@ -80,6 +90,9 @@ struct Master {
     std::vector<T> vw;          // DANA: N x d, row i = v^i, worker i's momentum
     std::vector<T> vsum;        // DANA: sum_j v^j
     int dana_sum = 1;           // 1 running sum, 0 summed afresh at every send
+    std::vector<T> v2;          // Adam: second moment (the first moment lives in v; gamma is beta_1)
+    T beta2 = (T)0.999f;        // Adam: beta_2
+    T adam_eps = (T)1e-8f;      // Adam: epsilon
     std::vector<int64_t> iter;  // iteration array of the SA algorithm
     int64_t k_done = 0;         // arrivals applied so far
     int64_t k_c = 0;            // refreshes of m so far
@@ -106,12 +119,64 @@ struct Master {
         for (int i = 0; i < n_workers; ++i) iter[i] = 0;
         k_done = 0;
         k_c = 0;
+        std::fill(v2.begin(), v2.end(), (T)0);
         std::fill(vw.begin(), vw.end(), (T)0);
         std::fill(vsum.begin(), vsum.end(), (T)0);
     }
 
     bool is_dana() const { return variant == DANA || variant == DANA_SA || variant == DANA_GA; }
-    bool has_gap() const { return variant == GA || variant == DANA_GA; }
+    bool has_gap() const { return variant == GA || variant == DANA_GA || variant == ADAM_GA; }
+    bool is_adam() const { return variant == ADAM || variant == ADAM_SA || variant == ADAM_GA; }
+
+    // One arrival of the three Adam masters. v holds the first moment, gamma is beta_1.
+    void push_adam(int i, const float* grad, int64_t k, int64_t tau) {
+        const T* s = &saved[(size_t)i * d];
+        const T beta1 = gamma;
+        const T one_minus_beta1 = (T)(1.0 - (double)beta1);
+        const T one_minus_beta2 = (T)(1.0 - (double)beta2);
+        const T one_minus_beta = (T)(1.0 - (double)beta);
+        const T inv_bias1 = (T)(1.0 / (1.0 - std::pow((double)beta1, (double)k)));
+        const T inv_bias2 = (T)(1.0 / (1.0 - std::pow((double)beta2, (double)k)));
+        double sum_gap = 0.0, max_gap = 0.0;
+        if (variant == ADAM_GA && c_order == 1) {
+            for (int64_t j = 0; j < d; ++j) {
+                const T g = (T)grad[j];
+                m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));
+            }
+            k_c += 1;
+        }
+        const T ib = k_c > 0 ? inv_bias() : (T)0;
+        for (int64_t j = 0; j < d; ++j) {
+            const T g = (T)grad[j];
+            T first;                                         // what is added to beta_1 m
+            if (variant == ADAM) {
+                first = one_minus_beta1 * g;
+            } else if (variant == ADAM_SA) {
+                first = one_minus_beta1 * (g / (T)tau);      // (1 - beta_1) g / tau
+            } else {
+                const T C = coeff(m[j], ib);
+                const T dist = std::fabs(theta[j] - s[j]);
+                const T G = dist / C + (T)1;
+                first = (one_minus_beta1 / G) * g;           // ((1 - beta_1) / G) (.) g
+                sum_gap += (double)G;
+                if ((double)G > max_gap) max_gap = (double)G;
+            }
+            v[j] = std::fma(beta1, v[j], first);
+            v2[j] = std::fma(beta2, v2[j], one_minus_beta2 * (g * g));
+            const T m_hat = v[j] * inv_bias1;
+            const T v_hat = v2[j] * inv_bias2;
+            theta[j] = theta[j] - (eta * m_hat) / (std::sqrt(v_hat) + adam_eps);
+        }
+        if (variant == ADAM_GA && c_order == 0) {
+            for (int64_t j = 0; j < d; ++j) {
+                const T g = (T)grad[j];
+                m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));
+            }
+            k_c += 1;
+        }
+        last_sum_gap = sum_gap;
+        last_max_gap = max_gap;
+    }
 
     void pull(int i) {
         if (is_dana()) { pull_dana(i); return; }
@@ -182,6 +247,8 @@ struct Master {
         const T* s = &saved[(size_t)i * d];
         if (is_dana()) {
             push_dana(i, grad, tau);
+        } else if (is_adam()) {
+            push_adam(i, grad, k, tau);
         } else if (variant == SA_GRAD) {
             for (int64_t j = 0; j < d; ++j) {
                 const T g_tau = (T)grad[j] / (T)tau;
@@ -241,6 +308,9 @@ struct Master {
     void set_state(const double* th, const double* vv, const double* mm, const double* sv,
                    const int64_t* it, int64_t kd, int64_t kc, const double* vworkers) {
         for (int64_t j = 0; j < d; ++j) { theta[j] = (T)th[j]; v[j] = (T)vv[j]; m[j] = (T)mm[j]; }
+        if (is_adam()) {      // vworkers carries Adam's second moment (one row)
+            for (int64_t j = 0; j < d; ++j) v2[j] = (T)vworkers[j];
+        }
         if (is_dana()) {      // vv carries sum_j v^j, vworkers the N rows
             for (int64_t j = 0; j < d; ++j) vsum[j] = (T)vv[j];
             for (size_t q = 0; q < (size_t)n_workers * d; ++q) vw[q] = (T)vworkers[q];
@@ -285,6 +355,7 @@ Master<T>* make(int64_t d, int n, double lr, double momentum, double beta, int v
     M->m.assign(d, 0);
     M->saved.assign((size_t)n * d, 0);
     M->iter.assign(n, 0);
+    if (M->is_adam()) M->v2.assign(d, 0);
     if (M->is_dana()) {
         M->vw.assign((size_t)n * d, 0);
         M->vsum.assign(d, 0);
@@ -301,7 +372,7 @@ extern "C" {
 void* gao_create(int64_t d, int n_workers, double lr, double momentum, double beta, int variant,
                  int precision) {
     if (d <= 0 || n_workers <= 0 || (precision != 32 && precision != 64)) return nullptr;
-    if (variant < 0 || variant > 6) return nullptr;
+    if (variant < 0 || variant > 9) return nullptr;
     auto* h = new (std::nothrow) Handle{precision, nullptr, nullptr};
     if (!h) return nullptr;
     try {
@@ -344,6 +415,11 @@ void gao_set_state(void* p, const double* th, const double* v, const double* m, 
     auto* h = (Handle*)p;
     DISPATCH(h, set_state(th, v, m, saved, iter, k_done, k_c, v_workers));
 }
+void gao_set_adam(void* p, double beta2, double adam_eps) {
+    auto* h = (Handle*)p;
+    if (h->precision == 32) { h->f->beta2 = (float)beta2; h->f->adam_eps = (float)adam_eps; }
+    else { h->g->beta2 = (double)(float)beta2; h->g->adam_eps = (double)(float)adam_eps; }
+}
 void gao_set_dana_sum(void* p, int mode) {
     auto* h = (Handle*)p;
     if (h->precision == 32) h->f->dana_sum = mode; else h->g->dana_sum = mode;
@@ -357,7 +433,8 @@ void gao_stats(void* p, double* sum_gap, double* max_gap) {
 }
 
 // which: 0 theta, 1 v (DANA: sum_j v^j), 2 m, 3 C (derived from m), 4+i saved copy of worker i,
-// 100000+i worker i's momentum v^i (DANA). Output in double.
+// 100000+i worker i's momentum v^i (DANA), 200000 Adam's second moment (its first is 1).
+// Output in double.
 int gao_get(void* p, int which, double* out) {
     auto* h = (Handle*)p;
     auto copy = [&](auto* M) -> int {
@@ -366,6 +443,7 @@ int gao_get(void* p, int which, double* out) {
         else if (which == 1 && M->is_dana()) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->vsum[j];
         else if (which >= 100000 && which < 100000 + M->n_workers && M->is_dana())
             for (int64_t j = 0; j < d; ++j) out[j] = (double)M->vw[(size_t)(which - 100000) * d + j];
+        else if (which == 200000 && M->is_adam()) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->v2[j];
         else if (which == 1) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->v[j];
         else if (which == 2) for (int64_t j = 0; j < d; ++j) out[j] = (double)M->m[j];
         else if (which == 3) {

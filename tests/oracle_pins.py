@@ -11,7 +11,7 @@ from fractions import Fraction
 
 import numpy as np
 
-ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA = range(7)
+ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA, ADAM, ADAM_SA, ADAM_GA = range(10)
 THETA, V, M, C = 0, 1, 2, 3
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
@@ -606,6 +606,174 @@ def pin_dana_exact_brute_force(make):
                         assert np.all(np.abs(got - want) <= tol * (1 + np.abs(want))), (variant, c_order, prec)
 
 
+# ------------------------------------------------------------------ Adam masters
+def pin_adam_is_torch_adam(make):
+    """Algorithm 'Adam: master' ignores staleness altogether: whatever the schedule it is the
+    textbook Adam, checked against torch.optim.Adam; its first step moves every parameter by
+    eta * g / (|g| + eps)."""
+    import torch
+    d, eta, b1, b2, eps = 29, 0.01, 0.9, 0.999, 1e-8
+    r = _rng(31)
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 2, 0, 2, 1, 1, 0, 2, 2, 0, 1]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    o = make(d, 3, eta, b1, 0.999, ADAM, precision=64, beta2=b2, adam_eps=eps)
+    o.set_params(th0)
+    p = torch.tensor(th0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([p], lr=float(np.float32(eta)), betas=(float(np.float32(b1)), float(np.float32(b2))),
+                           eps=float(np.float32(eps)))
+    for k, (i, g) in enumerate(zip(sched, grads)):
+        o.push(i, g)
+        o.pull(i)
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        if k == 0:
+            g64 = g.astype(np.float64)
+            step1 = float(np.float32(eta)) * g64 / (np.abs(g64) + float(np.float32(eps)))
+            assert np.allclose(o.get(THETA), th0.astype(np.float64) - step1, rtol=1e-12, atol=1e-14)
+        assert np.allclose(o.get(THETA), p.detach().numpy(), rtol=1e-10, atol=1e-12), k
+    st = opt.state[p]
+    assert np.allclose(o.get(V), st["exp_avg"].numpy(), rtol=1e-12, atol=1e-15)
+    assert np.allclose(o.second_moment(), st["exp_avg_sq"].numpy(), rtol=1e-12, atol=1e-18)
+    o32 = make(d, 3, eta, b1, 0.999, ADAM, precision=32, beta2=b2, adam_eps=eps)
+    o32.set_params(th0)
+    o32.push_batch(sched, grads)
+    assert np.allclose(o32.get(THETA), p.detach().numpy(), rtol=1e-4, atol=1e-5)
+
+
+def pin_adam_penalty_on_first_moment_only(make):
+    """Algorithms 'Adam-Staleness-Aware' and 'Adam-Gap-Aware': the second moment is that of
+    plain Adam, bit for bit; the first moment accumulates (1-beta1) g / tau (SA), resp.
+    ((1-beta1)/G) g (GA). One worker (tau = 1) makes Adam-SA plain Adam; where the master still
+    equals the saved copy Adam-GA adds exactly (1-beta1) g."""
+    d, n, eta, b1 = 16, 3, 0.01, 0.9
+    r = _rng(32)
+    th0 = _f32(r.normal(size=d))
+    sched, want_tau = [0, 1, 2, 0, 2], [1, 2, 3, 3, 2]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    runs = {}
+    for variant in (ADAM, ADAM_SA, ADAM_GA):
+        o = make(d, n, eta, b1, 0.999, variant, precision=64)
+        o.set_params(th0)
+        assert o.push_batch(sched, grads) == want_tau
+        runs[variant] = o
+    for variant in (ADAM_SA, ADAM_GA):
+        assert np.array_equal(runs[variant].second_moment(), runs[ADAM].second_moment())
+    B1 = float(np.float32(b1))
+    m_sa = np.zeros(d)
+    for g, tau in zip(grads, want_tau):
+        m_sa = B1 * m_sa + (1 - B1) * g.astype(np.float64) / tau
+    assert np.allclose(runs[ADAM_SA].get(V), m_sa, rtol=1e-12, atol=1e-16)
+    assert not np.allclose(runs[ADAM_SA].get(V), runs[ADAM].get(V), rtol=1e-3)
+    # one worker: every delay is 1
+    a = make(d, 1, eta, b1, 0.999, ADAM_SA, precision=32)
+    b = make(d, 1, eta, b1, 0.999, ADAM, precision=32)
+    for o in (a, b):
+        o.set_params(th0)
+        o.push_batch([0] * 5, grads)
+    assert np.array_equal(a.get(THETA), b.get(THETA))
+    # Adam-GA, first arrival of each worker's untouched elements: G = 1 there
+    g1 = grads[0].copy()
+    g1[1::2] = 0.0
+    ga = make(d, 2, eta, b1, 0.999, ADAM_GA, precision=32)
+    ad = make(d, 2, eta, b1, 0.999, ADAM, precision=32)
+    for o in (ga, ad):
+        o.set_params(th0)
+        o.push(1, g1)
+        o.pull(1)
+    G = ga.gap(0)
+    assert np.all(G[1::2] == 1.0) and np.all(G[0::2] > 1.0)
+    for o in (ga, ad):
+        o.push(0, grads[1])
+    assert np.array_equal(ga.get(V)[1::2], ad.get(V)[1::2])
+    assert np.array_equal(ga.get(THETA)[1::2], ad.get(THETA)[1::2])
+    # penalised elements: first moment is beta1 m + ((1-beta1)/G) g with the G read before the push
+    m_prev = (1 - B1) * g1.astype(np.float64)
+    want = B1 * m_prev + (1 - B1) / G * grads[1].astype(np.float64)
+    assert np.allclose(ga.get(V), want, rtol=1e-5, atol=1e-9)
+
+
+def pin_adam_ga_coefficient(make):
+    """Adam-GA's C: the C algorithm with gamma = 0. A gradient of constant magnitude c gives
+    C = eta_max (c + eps) from the first refresh on, whatever Adam's own moments do."""
+    d, eta = 12, 0.01
+    c = _f32(np.linspace(0.02, 2.0, d))
+    for c_order in (0, 1):
+        o = make(d, 1, eta, 0.9, 0.999, ADAM_GA, precision=64, c_order=c_order)
+        o.set_params(np.zeros(d, np.float32))
+        sign = 1.0
+        for k in range(1, 25):
+            sign = -sign if k % 4 == 0 else sign
+            o.push(0, _f32(c * sign))
+            o.pull(0)
+            assert np.allclose(o.get(C), float(np.float32(eta)) * (c.astype(np.float64) + 1e-8), rtol=1e-11)
+
+
+def brute_force_adam(th0, sched, grads, n, eta, b1, b2, eps_adam, beta, eps, variant, c_order):
+    d = len(th0)
+    th = [Fraction(float(x)) for x in th0]
+    m1 = [Fraction(0)] * d
+    v2 = [Fraction(0)] * d
+    mc = [Fraction(0)] * d
+    saved = [list(th) for _ in range(n)]
+    it = [0] * n
+    refreshes = 0
+    taus = []
+    for k, (i, g) in enumerate(zip(sched, grads), start=1):
+        g = [Fraction(float(x)) for x in g]
+        tau = k - it[i]
+        taus.append(tau)
+        for j in range(d):
+            if variant == ADAM:
+                first = (1 - b1) * g[j]
+            elif variant == ADAM_SA:
+                first = (1 - b1) * g[j] / tau
+            else:
+                r, mj = refreshes, mc[j]
+                if c_order == 1:
+                    mj = beta * mj + (1 - beta) * g[j] * g[j]
+                    r += 1
+                    mc[j] = mj
+                Cj = eta * eps if r == 0 else eta * (_sqrt_fraction(mj / (1 - beta ** r)) + eps)
+                Gj = abs(th[j] - saved[i][j]) / Cj + 1
+                first = (1 - b1) / Gj * g[j]
+                if c_order == 0:
+                    mc[j] = beta * mc[j] + (1 - beta) * g[j] * g[j]
+            m1[j] = b1 * m1[j] + first
+            v2[j] = b2 * v2[j] + (1 - b2) * g[j] * g[j]
+            m_hat = m1[j] / (1 - b1 ** k)
+            v_hat = v2[j] / (1 - b2 ** k)
+            th[j] = th[j] - eta * m_hat / (_sqrt_fraction(v_hat) + eps_adam)
+        if variant == ADAM_GA:
+            refreshes += 1
+        saved[i] = list(th)
+        it[i] = k
+    return th, m1, v2, mc, taus
+
+
+def pin_adam_exact_brute_force(make):
+    """Algorithms 'Adam', 'Adam-Staleness-Aware', 'Adam-Gap-Aware: master' in exact arithmetic."""
+    r = _rng(33)
+    d, n = 3, 3
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 0, 2, 1, 0]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    eta, b1, b2, beta, eps = 0.0625, 0.75, 0.875, 0.9375, 2.0 ** -20
+    F = Fraction
+    for variant in (ADAM, ADAM_SA, ADAM_GA):
+        for c_order in ((0, 1) if variant == ADAM_GA else (0,)):
+            th, m1, v2, mc, taus = brute_force_adam(th0, sched, grads, n, F(eta), F(b1), F(b2), F(eps), F(beta),
+                                                    F(eps), variant, c_order)
+            for prec, tol in ((64, 5e-13), (32, 5e-5)):
+                o = make(d, n, eta, b1, beta, variant, precision=prec, c_order=c_order, eps=eps, beta2=b2,
+                         adam_eps=eps)
+                o.set_params(th0)
+                assert o.push_batch(sched, grads) == taus
+                for got, ref in ((o.get(THETA), th), (o.get(V), m1), (o.second_moment(), v2), (o.get(M), mc)):
+                    want = np.array([float(x) for x in ref])
+                    assert np.all(np.abs(got - want) <= tol * (1 + np.abs(want))), (variant, c_order, prec)
+
+
 ALL_PINS = [
     pin_gap_is_one_where_copy_equals_master,
     pin_one_worker_is_heavy_ball,
@@ -624,4 +792,8 @@ ALL_PINS = [
     pin_dana_structure,
     pin_dana_gap,
     pin_dana_exact_brute_force,
+    pin_adam_is_torch_adam,
+    pin_adam_penalty_on_first_moment_only,
+    pin_adam_ga_coefficient,
+    pin_adam_exact_brute_force,
 ]

@@ -77,6 +77,22 @@ MUTANTS = [
      "const T G = dist / C;\n                const T inv_gap = (T)1 / G;\n                g_pen"),
     ("dana_ga_m_from_sum", "m[j] = std::fma(beta, m[j], one_minus_beta * (vi[j] * vi[j]));",
      "m[j] = std::fma(beta, m[j], one_minus_beta * (vsum[j] * vsum[j]));"),
+    # the Adam masters
+    ("adam_first_moment_weight", "first = one_minus_beta1 * g;", "first = g;"),
+    ("adam_second_moment_of_penalised", "v2[j] = std::fma(beta2, v2[j], one_minus_beta2 * (g * g));",
+     "v2[j] = std::fma(beta2, v2[j], one_minus_beta2 * (first * first));"),
+    ("adam_second_moment_unsquared", "v2[j] = std::fma(beta2, v2[j], one_minus_beta2 * (g * g));",
+     "v2[j] = std::fma(beta2, v2[j], one_minus_beta2 * std::fabs(g));"),
+    ("adam_no_bias_correction_1", "const T m_hat = v[j] * inv_bias1;", "const T m_hat = v[j];"),
+    ("adam_no_bias_correction_2", "const T v_hat = v2[j] * inv_bias2;", "const T v_hat = v2[j];"),
+    ("adam_bias_exponent", "std::pow((double)beta1, (double)k)", "std::pow((double)beta1, (double)(k + 1))"),
+    ("adam_eps_inside_root", "(std::sqrt(v_hat) + adam_eps)", "std::sqrt(v_hat + adam_eps)"),
+    ("adam_step_sign", "theta[j] = theta[j] - (eta * m_hat)", "theta[j] = theta[j] + (eta * m_hat)"),
+    ("adam_sa_multiplies", "first = one_minus_beta1 * (g / (T)tau);", "first = one_minus_beta1 * (g * (T)tau);"),
+    ("adam_ga_divides_twice", "first = (one_minus_beta1 / G) * g;", "first = (one_minus_beta1 / G / G) * g;"),
+    ("adam_ga_unpenalised", "first = (one_minus_beta1 / G) * g;", "first = one_minus_beta1 * g;"),
+    ("adam_ga_c_from_first_moment", "m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));\n            }\n            k_c += 1;\n        }\n        last_sum_gap",
+     "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));\n            }\n            k_c += 1;\n        }\n        last_sum_gap"),
     ("dana_pull_forgets_iteration", "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);\n        }\n        iter[i] = k_done;",
      "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);\n        }"),
 ]
