@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--config", default="C5")
     ap.add_argument("--params", type=int, default=0, help="profiling aid: a one-segment vector of this size")
     ap.add_argument("--workers", type=int, default=32)
-    ap.add_argument("--variant", default="GA", choices=["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA"])
+    ap.add_argument("--variant", default="GA", choices=["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA", "ADAM", "ADAM_SA", "ADAM_GA"])
     ap.add_argument("--window", type=int, default=16)
     ap.add_argument("--math", default="exact", choices=["exact", "fast"])
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -58,8 +58,11 @@ def parse_args():
 def bytes_per_param_window(variant, k):
     """Algorithmic bytes one parameter moves in a k-arrival window (fp32): theta, v (and m) in
     and out once; per arrival the gradient (and, for GA, the saved copy) in and the saved copy out."""
-    state = 24 if variant in ("GA", "DANA_GA") else 16          # theta, v or sum_j v^j (, m) in and out
-    per_arrival = 8 + (4 if variant in ("GA", "DANA_GA") else 0)  # gradient in, sent copy out (, saved copy in)
+    gap = variant in ("GA", "DANA_GA", "ADAM_GA")
+    state = 24 if gap else 16                  # theta, v or sum_j v^j or Adam's m (, m behind C) in and out
+    if variant.startswith("ADAM"):
+        state += 8                             # Adam's second moment in and out
+    per_arrival = 8 + (4 if gap else 0)        # gradient in, sent copy out (, saved copy in)
     if variant.startswith("DANA"):
         per_arrival += 8                                           # the worker's v^i in and out
     return state + per_arrival * k

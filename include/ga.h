@@ -49,13 +49,21 @@ enum {
      * array of device memory. */
     GA_DANA = 4,    /* v^i <- gamma v^i + g                                   */
     GA_DANA_SA = 5, /* v^i <- gamma v^i + g / tau                             */
-    GA_DANA_GA = 6  /* v^i <- gamma v^i + (1/G) g, Gap against the saved estimate */
+    GA_DANA_GA = 6, /* v^i <- gamma v^i + (1/G) g, Gap against the saved estimate */
+    /* The Adam masters (appendix, Algorithms "Adam: master", "Adam-Staleness-Aware: master",
+     * "Adam-Gap-Aware: master"). `momentum` of ga_create is beta_1; beta_2 and Adam's epsilon are
+     * options (defaults 0.999, 1e-8). The penalty enters the first moment only. For Adam-GA the
+     * C algorithm is run with gamma = 0, i.e. on the raw gradient, with c_beta. */
+    GA_ADAM = 7,    /* m <- beta1 m + (1-beta1) g                         */
+    GA_ADAM_SA = 8, /* m <- beta1 m + (1-beta1) g / tau                   */
+    GA_ADAM_GA = 9  /* m <- beta1 m + ((1-beta1)/G) g                     */
 };
 
 enum { GA_OK = 0, GA_ERR_ARG = -1, GA_ERR_STATE = -2, GA_ERR_OOM = -3, GA_ERR_CUDA = -4 };
 
-/* vectors readable with ga_get; GA_V is the master's momentum v, or sum_j v^j for the DANA variants */
-enum { GA_THETA = 0, GA_V = 1, GA_M = 2, GA_C = 3 };
+/* vectors readable with ga_get; GA_V is the master's momentum v, sum_j v^j for the DANA variants,
+ * Adam's first moment for the Adam variants; GA_V2 is Adam's second moment */
+enum { GA_THETA = 0, GA_V = 1, GA_M = 2, GA_C = 3, GA_V2 = 4 };
 
 /* options for ga_set_option */
 enum {
@@ -69,8 +77,10 @@ enum {
     GA_OPT_STATS = 2,   /* 1: every GA push also reduces sum and max of the Gap over all
                            parameters (the quantity the paper logs per epoch, Appendix
                            "Gap and Delay"); read with ga_get_stats. Default 0. */
-    GA_OPT_WINDOW = 3   /* 1..16 (default 16): most arrivals fused into one launch by
+    GA_OPT_WINDOW = 3,  /* 1..16 (default 16): most arrivals fused into one launch by
                            ga_push_batch. */
+    GA_OPT_ADAM_BETA2 = 4, /* Adam variants: beta_2 in [0,1), default 0.999; before the first arrival */
+    GA_OPT_ADAM_EPS = 5    /* Adam variants: epsilon > 0, default 1e-8; before the first arrival */
 };
 
 #define GA_MAX_WINDOW 16

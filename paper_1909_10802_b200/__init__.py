@@ -15,14 +15,16 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("GA_LIBRARY") or os.path.join(_HERE, "libga.so")   # GA_LIBRARY: another build
 
-GA_ASGD, GA_SA, GA_GA, GA_SA_GRAD, GA_DANA, GA_DANA_SA, GA_DANA_GA = range(7)
+(GA_ASGD, GA_SA, GA_GA, GA_SA_GRAD, GA_DANA, GA_DANA_SA, GA_DANA_GA, GA_ADAM, GA_ADAM_SA,
+ GA_ADAM_GA) = range(10)
 GA_OK, GA_ERR_ARG, GA_ERR_STATE, GA_ERR_OOM, GA_ERR_CUDA = 0, -1, -2, -3, -4
-GA_THETA, GA_V, GA_M, GA_C = 0, 1, 2, 3
-GA_OPT_C_ORDER, GA_OPT_MATH, GA_OPT_STATS, GA_OPT_WINDOW = 0, 1, 2, 3
+GA_THETA, GA_V, GA_M, GA_C, GA_V2 = 0, 1, 2, 3, 4
+GA_OPT_C_ORDER, GA_OPT_MATH, GA_OPT_STATS, GA_OPT_WINDOW, GA_OPT_ADAM_BETA2, GA_OPT_ADAM_EPS = range(6)
 GA_MAX_WINDOW = 16
 GA_NOALLOC_MAX_PARAMS = 1 << 28
 VARIANTS = {"ASGD": GA_ASGD, "SA": GA_SA, "GA": GA_GA, "SA_GRAD": GA_SA_GRAD, "DANA": GA_DANA,
-            "DANA_SA": GA_DANA_SA, "DANA_GA": GA_DANA_GA}
+            "DANA_SA": GA_DANA_SA, "DANA_GA": GA_DANA_GA, "ADAM": GA_ADAM, "ADAM_SA": GA_ADAM_SA,
+            "ADAM_GA": GA_ADAM_GA}
 
 # every symbol include/ga.h declares: name -> (restype, argtypes)
 _c = ctypes
@@ -252,7 +254,7 @@ class Engine:
 
 
 # ---- checkpoint blobs (layout of ga_export_state): header, iter[N], theta, v, m, saved[N][d]
-_HEADER = "<IIqqqqffffiiiiii"
+_HEADER = "<IIqqqqffffiiiiiiff"
 _MAGIC = 0x47415331
 
 
@@ -263,16 +265,18 @@ def unpack_state(blob):
     import numpy as np
     hs = struct.calcsize(_HEADER)
     (magic, version, d, n, k_done, k_c, lr, gamma, beta, eps, variant, c_order, fast_math, stats,
-     window, _) = struct.unpack_from(_HEADER, blob, 0)
-    if magic != _MAGIC or version != 1:
+     window, _, beta2, adam_eps) = struct.unpack_from(_HEADER, blob, 0)
+    if magic != _MAGIC or version != 2:
         raise ValueError("not a Gap-Aware master checkpoint")
     off = hs
     iters = np.frombuffer(blob, dtype=np.int64, count=n, offset=off).copy()
     off += 8 * n
     dana = variant in (GA_DANA, GA_DANA_SA, GA_DANA_GA)
-    rows = 3 + n * (2 if dana else 1)
+    adam = variant in (GA_ADAM, GA_ADAM_SA, GA_ADAM_GA)
+    rows = 3 + n * (2 if dana else 1) + (1 if adam else 0)
     vecs = np.frombuffer(blob, dtype=np.float32, count=rows * d, offset=off).reshape(rows, d).copy()
-    extra = {"v_workers": vecs[3 + n:]} if dana else {}
+    extra = {"v_workers": vecs[3 + n:]} if dana else {"v2": vecs[3 + n]} if adam else {}
+    extra.update(beta2=beta2, adam_eps=adam_eps)
     return dict(**extra, d=d, n_workers=n, k_done=k_done, k_c=k_c, lr=lr, momentum=gamma, c_beta=beta, eps=eps,
                 variant=variant, c_order=c_order, fast_math=fast_math, stats=stats, window=window,
                 iter=iters, theta=vecs[0], v=vecs[1], m=vecs[2], saved=vecs[3:3 + n])
@@ -283,11 +287,12 @@ def pack_state(st):
     import struct
 
     import numpy as np
-    head = struct.pack(_HEADER, _MAGIC, 1, st["d"], st["n_workers"], st["k_done"], st["k_c"], st["lr"],
+    head = struct.pack(_HEADER, _MAGIC, 2, st["d"], st["n_workers"], st["k_done"], st["k_c"], st["lr"],
                        st["momentum"], st["c_beta"], st["eps"], st["variant"], st["c_order"],
-                       st["fast_math"], st["stats"], st["window"], 0)
+                       st["fast_math"], st["stats"], st["window"], 0, st.get("beta2", 0.999),
+                       st.get("adam_eps", 1e-8))
     parts = [head, np.ascontiguousarray(st["iter"], dtype=np.int64).tobytes()]
-    for name in ("theta", "v", "m", "saved") + (("v_workers",) if "v_workers" in st else ()):
+    for name in ("theta", "v", "m", "saved") + tuple(x for x in ("v_workers", "v2") if x in st):
         a = np.ascontiguousarray(st[name], dtype=np.float32)
         parts.append(a.tobytes())
     return b"".join(parts)

@@ -41,6 +41,8 @@ struct ga_engine {
     int c_order = 0, fast_math = 0, stats = 0, window = GA_MAX_WINDOW;
     float *theta = nullptr, *vel = nullptr, *mom = nullptr, *saved = nullptr;
     float* vworker = nullptr;     // DANA: N rows, v^i of every worker (vel then holds their sum)
+    float* sec = nullptr;         // Adam: second moment (vel holds the first moment, gamma is beta_1)
+    float beta2 = 0.999f, adam_eps = 1e-8f;
     std::vector<int64_t> iter;
     int64_t k_done = 0, k_c = 0;
     cudaStream_t stream = nullptr;
@@ -62,8 +64,9 @@ struct ga_engine {
     float* row(int i) const { return saved + (size_t)i * stride; }
     float* vrow(int i) const { return vworker ? vworker + (size_t)i * stride : nullptr; }
     bool is_dana() const { return variant == GA_DANA || variant == GA_DANA_SA || variant == GA_DANA_GA; }
-    bool is_gap() const { return variant == GA_GA || variant == GA_DANA_GA; }
-    bool is_tau_grad() const { return variant == GA_SA_GRAD || variant == GA_DANA_SA; }
+    bool is_adam() const { return variant == GA_ADAM || variant == GA_ADAM_SA || variant == GA_ADAM_GA; }
+    bool is_gap() const { return variant == GA_GA || variant == GA_DANA_GA || variant == GA_ADAM_GA; }
+    bool is_tau_grad() const { return variant == GA_SA_GRAD || variant == GA_DANA_SA || variant == GA_ADAM_SA; }
     ga::Hyper hyper() const {
         ga::Hyper h;
         h.eta_max = lr;
@@ -72,6 +75,10 @@ struct ga_engine {
         h.one_minus_beta = (float)(1.0 - (double)beta);
         h.eps = eps;
         h.eta_gamma = lr * gamma;
+        h.one_minus_gamma = (float)(1.0 - (double)gamma);
+        h.beta2 = beta2;
+        h.one_minus_beta2 = (float)(1.0 - (double)beta2);
+        h.adam_eps = adam_eps;
         return h;
     }
     // 1/(1-beta^k) for the C in force after k refreshes of m; 0 before the first (C = eta_max*eps)
@@ -147,10 +154,10 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
     // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner
     if (w.K == 1)
         ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, 1><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
-            e->theta, e->vel, e->mom, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
+            e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
     else
         ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, GA_WINDOW_BATCH><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
-            e->theta, e->vel, e->mom, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
+            e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
     if (STATS) {
         ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev);
     }
@@ -159,7 +166,7 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
 template <int FAMILY>
 void launch_family(ga_engine* e, const ga::Window& w, long long vb, long long ve, cudaStream_t st, bool stats) {
     if (e->is_gap()) {
-        const bool exact = !e->fast_math;
+        const bool exact = !e->fast_math || FAMILY == ga::ADAM;   // Adam has no fast-math form
 #define GA_CASE(EX, CO, ST) launch_window_t<FAMILY, ga::PEN_GAP, EX, CO, ST>(e, w, vb, ve, st)
         if (exact) {
             if (e->c_order == 0) { if (stats) GA_CASE(true, 0, true); else GA_CASE(true, 0, false); }
@@ -181,6 +188,7 @@ int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long l
     if (vec_end <= vec_begin || w.K <= 0) return GA_OK;
     const bool stats = allow_stats && e->stats && e->is_gap();
     if (e->is_dana()) launch_family<ga::DANA>(e, w, vec_begin, vec_end, st, stats);
+    else if (e->is_adam()) launch_family<ga::ADAM>(e, w, vec_begin, vec_end, st, stats);
     else launch_family<ga::MOM>(e, w, vec_begin, vec_end, st, stats);
     GA_CUDA(e, cudaGetLastError());
     if (stats) { e->stats_valid = true; e->stats_slot = w.K - 1; }
@@ -202,6 +210,11 @@ void fill_window(ga_engine* e, ga::Window& w, const int* workers, const float* c
         w.saved[j] = e->row(i);
         w.vworker[j] = e->vrow(i);
         w.tau[j] = (float)tau;
+        w.bias1[j] = w.bias2[j] = 1.f;
+        if (e->is_adam()) {   // Adam's bias corrections use the arrival index
+            w.bias1[j] = (float)(1.0 / (1.0 - std::pow((double)e->gamma, (double)k)));
+            w.bias2[j] = (float)(1.0 / (1.0 - std::pow((double)e->beta2, (double)k)));
+        }
         w.eta_eff[j] = e->variant == GA_SA ? e->lr / (float)tau : e->lr;
         if (e->is_gap()) {
             // the C in force for this arrival: after k_c refreshes (lagged order), or after
@@ -219,6 +232,7 @@ void fill_window(ga_engine* e, ga::Window& w, const int* workers, const float* c
         w.saved[j] = nullptr;
         w.vworker[j] = nullptr;
         w.tau[j] = 1.f;
+        w.bias1[j] = w.bias2[j] = 1.f;
         w.inv_bias[j] = 0.f;
         w.eta_eff[j] = 0.f;
     }
@@ -280,7 +294,7 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
     if (!(lr > 0.f) || !std::isfinite(lr)) { fail(GA_ERR_ARG, "lr must be positive and finite"); return nullptr; }
     if (!(std::fabs(momentum) < 1.f)) { fail(GA_ERR_ARG, "|momentum| must be < 1"); return nullptr; }
     if (!(c_beta >= 0.f && c_beta < 1.f)) { fail(GA_ERR_ARG, "c_beta must be in [0, 1)"); return nullptr; }
-    if (variant < GA_ASGD || variant > GA_DANA_GA) { fail(GA_ERR_ARG, "unknown variant %d", variant); return nullptr; }
+    if (variant < GA_ASGD || variant > GA_ADAM_GA) { fail(GA_ERR_ARG, "unknown variant %d", variant); return nullptr; }
     ga_engine* e = new (std::nothrow) ga_engine();
     if (!e) { fail(GA_ERR_OOM, "out of host memory"); return nullptr; }
     e->d = (long long)n_params;
@@ -307,13 +321,15 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
               cudaMalloc(&e->partials, sizeof(ga::StatsPartial) * (size_t)e->stats_blocks * ga::kMaxWindow) == cudaSuccess &&
               cudaMalloc(&e->stats_dev, sizeof(double) * 2 * ga::kMaxWindow) == cudaSuccess &&
               cudaMalloc(&e->pull_err, sizeof(int)) == cudaSuccess &&
-              (!e->is_dana() || cudaMalloc(&e->vworker, row_bytes * (size_t)n_workers) == cudaSuccess);
+              (!e->is_dana() || cudaMalloc(&e->vworker, row_bytes * (size_t)n_workers) == cudaSuccess) &&
+              (!e->is_adam() || cudaMalloc(&e->sec, row_bytes) == cudaSuccess);
     if (ok) {
         ok = cudaMemset(e->theta, 0, row_bytes) == cudaSuccess && cudaMemset(e->vel, 0, row_bytes) == cudaSuccess &&
              cudaMemset(e->mom, 0, row_bytes) == cudaSuccess &&
              cudaMemset(e->saved, 0, row_bytes * (size_t)n_workers) == cudaSuccess &&
              cudaMemset(e->pull_err, 0, sizeof(int)) == cudaSuccess &&
              (!e->vworker || cudaMemset(e->vworker, 0, row_bytes * (size_t)n_workers) == cudaSuccess) &&
+             (!e->sec || cudaMemset(e->sec, 0, row_bytes) == cudaSuccess) &&
              cudaFuncSetAttribute(ga::ga_pull_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   ga::kPullStages * ga::kPullChunk) == cudaSuccess &&
              cudaDeviceSynchronize() == cudaSuccess;
@@ -336,6 +352,7 @@ void ga_destroy(ga_engine* e) {
     cudaFree(e->mom);
     cudaFree(e->saved);
     cudaFree(e->vworker);
+    cudaFree(e->sec);
     cudaFree(e->partials);
     cudaFree(e->stats_dev);
     cudaFree(e->pull_err);
@@ -364,6 +381,7 @@ int ga_set_params(ga_engine* e, const float* theta0_dev) {
     ga::ga_set_params_kernel<<<grid_1d(e->stride, 256, 148 * 8), 256, 0, e->stream>>>(
         theta0_dev, e->theta, e->vel, e->mom, e->saved, e->vworker, e->n_workers, e->d, e->stride);
     GA_CUDA(e, cudaGetLastError());
+    if (e->sec) GA_CUDA(e, cudaMemsetAsync(e->sec, 0, sizeof(float) * (size_t)e->stride, e->stream));
     std::fill(e->iter.begin(), e->iter.end(), 0);
     e->k_done = 0;
     e->k_c = 0;
@@ -490,6 +508,10 @@ int ga_get(ga_engine* e, int which, float* out_dev) {
     if (int rc = check_dev_ptr(out_dev, "out_dev")) return rc;
     DeviceGuard guard(e->device);
     const float* src = which == GA_THETA ? e->theta : which == GA_V ? e->vel : which == GA_M ? e->mom : nullptr;
+    if (which == GA_V2) {
+        if (!e->is_adam()) return fail(GA_ERR_STATE, "only the Adam variants keep a second moment");
+        src = e->sec;
+    }
     if (src) {
         GA_CUDA(e, cudaMemcpyAsync(out_dev, src, sizeof(float) * (size_t)e->d, cudaMemcpyDeviceToDevice, e->stream));
     } else if (which == GA_C) {
@@ -544,6 +566,16 @@ int ga_set_option(ga_engine* e, int key, double value) {
             e->stats = v;
             if (!v) e->stats_valid = false;
             return GA_OK;
+        case GA_OPT_ADAM_BETA2:
+            if (!(value >= 0.0 && value < 1.0)) return fail(GA_ERR_ARG, "GA_OPT_ADAM_BETA2 must be in [0, 1)");
+            if (e->k_done != 0) return fail(GA_ERR_STATE, "GA_OPT_ADAM_BETA2 can only change before the first arrival");
+            e->beta2 = (float)value;
+            return GA_OK;
+        case GA_OPT_ADAM_EPS:
+            if (!(value > 0.0)) return fail(GA_ERR_ARG, "GA_OPT_ADAM_EPS must be positive");
+            if (e->k_done != 0) return fail(GA_ERR_STATE, "GA_OPT_ADAM_EPS can only change before the first arrival");
+            e->adam_eps = (float)value;
+            return GA_OK;
         case GA_OPT_WINDOW:
             if (v < 1 || v > GA_MAX_WINDOW) return fail(GA_ERR_ARG, "GA_OPT_WINDOW must be in [1, %d]", GA_MAX_WINDOW);
             e->window = v;
@@ -583,17 +615,19 @@ struct StateHeader {
     int64_t d, n_workers, k_done, k_c;
     float lr, gamma, beta, eps;
     int32_t variant, c_order, fast_math, stats, window, reserved;
+    float beta2, adam_eps;
 };
 
 size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
     if (check_engine(e)) return 0;
     const size_t vec = sizeof(float) * (size_t)e->d;
-    const size_t rows = 3 + (size_t)e->n_workers * (e->is_dana() ? 2 : 1);
+    const size_t rows = 3 + (size_t)e->n_workers * (e->is_dana() ? 2 : 1) + (e->is_adam() ? 1 : 0);
     const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows;
     if (!buf_host || cap < need) return need;
     DeviceGuard guard(e->device);
     StateHeader h{};
-    h.magic = kStateMagic; h.version = 1;
+    h.magic = kStateMagic; h.version = 2;
+    h.beta2 = e->beta2; h.adam_eps = e->adam_eps;
     h.d = e->d; h.n_workers = e->n_workers; h.k_done = e->k_done; h.k_c = e->k_c;
     h.lr = e->lr; h.gamma = e->gamma; h.beta = e->beta; h.eps = e->eps;
     h.variant = e->variant; h.c_order = e->c_order; h.fast_math = e->fast_math; h.stats = e->stats; h.window = e->window;
@@ -608,6 +642,7 @@ size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
         err = cudaMemcpyAsync(p, e->row(i), vec, cudaMemcpyDeviceToHost, e->stream);
     for (int i = 0; e->is_dana() && i < e->n_workers && err == cudaSuccess; ++i, p += vec)
         err = cudaMemcpyAsync(p, e->vrow(i), vec, cudaMemcpyDeviceToHost, e->stream);
+    if (e->is_adam() && err == cudaSuccess) err = cudaMemcpyAsync(p, e->sec, vec, cudaMemcpyDeviceToHost, e->stream);
     if (err == cudaSuccess) err = cudaStreamSynchronize(e->stream);
     if (err != cudaSuccess) { cuda_fail(e, err, "ga_export_state"); return 0; }
     return need;
@@ -618,12 +653,12 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
     if (!buf_host || len < sizeof(StateHeader)) return fail(GA_ERR_ARG, "state buffer too short");
     StateHeader h;
     std::memcpy(&h, buf_host, sizeof h);
-    if (h.magic != kStateMagic || h.version != 1) return fail(GA_ERR_ARG, "not a state written by ga_export_state");
+    if (h.magic != kStateMagic || h.version != 2) return fail(GA_ERR_ARG, "not a state written by ga_export_state");
     if (h.d != e->d || h.n_workers != e->n_workers)
         return fail(GA_ERR_ARG, "state is for %lld parameters / %lld workers", (long long)h.d, (long long)h.n_workers);
     const size_t vec = sizeof(float) * (size_t)e->d;
     if (h.variant != e->variant) return fail(GA_ERR_ARG, "state is for variant %d, engine is variant %d", h.variant, e->variant);
-    const size_t rows = 3 + (size_t)e->n_workers * (e->is_dana() ? 2 : 1);
+    const size_t rows = 3 + (size_t)e->n_workers * (e->is_dana() ? 2 : 1) + (e->is_adam() ? 1 : 0);
     const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows;
     if (len < need) return fail(GA_ERR_ARG, "state buffer truncated");
     if ( h.window < 1 || h.window > GA_MAX_WINDOW || h.k_done < 0 || h.k_c < 0)
@@ -639,10 +674,12 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
         GA_CUDA(e, cudaMemcpyAsync(e->row(i), p, vec, cudaMemcpyHostToDevice, e->stream));
     for (int i = 0; e->is_dana() && i < e->n_workers; ++i, p += vec)
         GA_CUDA(e, cudaMemcpyAsync(e->vrow(i), p, vec, cudaMemcpyHostToDevice, e->stream));
+    if (e->is_adam()) GA_CUDA(e, cudaMemcpyAsync(e->sec, p, vec, cudaMemcpyHostToDevice, e->stream));
     GA_CUDA(e, cudaStreamSynchronize(e->stream));
     e->iter = iter;
     e->k_done = h.k_done; e->k_c = h.k_c;
     e->lr = h.lr; e->gamma = h.gamma; e->beta = h.beta; e->eps = h.eps;
+    e->beta2 = h.beta2; e->adam_eps = h.adam_eps;
     e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window;
     e->stats_valid = false;
     return GA_OK;
@@ -748,7 +785,8 @@ extern "C" int ga_gap_stats_noalloc(const float* theta_dev, const float* saved_d
     ga::StatsPartial* scratch = nullptr;
     if (int rc = noalloc_scratch(&scratch)) return rc;
     ga::Hyper h;
-    h.eta_max = lr_max; h.gamma = 0.f; h.eta_gamma = 0.f; h.beta = c_beta; h.one_minus_beta = (float)(1.0 - (double)c_beta); h.eps = 1e-8f;
+    h = ga::Hyper{};
+    h.eta_max = lr_max; h.beta = c_beta; h.one_minus_beta = (float)(1.0 - (double)c_beta); h.eps = 1e-8f;
     const float inv_bias = n_refreshes == 0 ? 0.f : (float)(1.0 / (1.0 - std::pow((double)c_beta, (double)n_refreshes)));
     const int blocks = (int)((n_params + kNoAllocTile - 1) / kNoAllocTile);
     cudaStream_t st = (cudaStream_t)cuda_stream;

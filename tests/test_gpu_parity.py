@@ -54,16 +54,19 @@ def _compare_engine(P, run, o, idx=None, label=""):
     import torch
     sel = None if idx is None else torch.as_tensor(idx, device="cuda")
     names = (("theta", P.GA_THETA, o.THETA), ("v", P.GA_V, o.V))
-    if run.engine.variant in (P.GA_GA, P.GA_DANA_GA):
+    if run.engine.variant in (P.GA_GA, P.GA_DANA_GA, P.GA_ADAM_GA):
         names += (("m", P.GA_M, o.M), ("C", P.GA_C, o.C))
+    if run.engine.variant in (P.GA_ADAM, P.GA_ADAM_SA, P.GA_ADAM_GA):
+        names += (("v2", ("v2", 0), None),)
     if run.engine.variant in (P.GA_DANA, P.GA_DANA_SA, P.GA_DANA_GA):
         names += tuple((f"v^{i}", ("vw", i), None) for i in range(run.engine.n_workers))
     names += tuple((f"sent^{i}", ("sent", i), None) for i in range(min(run.engine.n_workers, 8)))
     for name, which, owhich in names:
         if isinstance(which, tuple):
             kind, i = which
-            got = run.engine.get_worker_momentum(i) if kind == "vw" else run.engine.saved(i)
-            ref = o.worker_momentum(i) if kind == "vw" else o.saved(i)
+            got = (run.engine.get_worker_momentum(i) if kind == "vw" else
+                   run.engine.get(P.GA_V2) if kind == "v2" else run.engine.saved(i))
+            ref = o.worker_momentum(i) if kind == "vw" else o.second_moment() if kind == "v2" else o.saved(i)
         else:
             got = run.engine.get(which)
             ref = o.get(owhich)
@@ -105,7 +108,7 @@ def test_device_generator_sparse_rows_and_subrange(P):
 
 
 # ----------------------------------------------------------------------------- small, exhaustive
-ALL_VARIANTS = ["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA"]
+ALL_VARIANTS = ["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA", "ADAM", "ADAM_SA", "ADAM_GA"]
 
 
 @pytest.mark.parametrize("variant", ALL_VARIANTS)
@@ -113,7 +116,7 @@ ALL_VARIANTS = ["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA"]
 def test_mini_trajectory(P, variant, window):
     from paper_1909_10802_b200.runner import Run
     wl = W.config("mini")
-    for c_order in ((0, 1) if variant in ("GA", "DANA_GA") else (0,)):
+    for c_order in ((0, 1) if variant in ("GA", "DANA_GA", "ADAM_GA") else (0,)):
         run = Run(wl, variant, window, options={P.GA_OPT_C_ORDER: c_order})
         delays = run.run()
         o, odelays, _ = run_oracle(wl, variant, c_order=c_order)
@@ -189,8 +192,8 @@ def test_c3_window_invariance(P):
         torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("variant", ["DANA_GA", "DANA", "DANA_SA", "SA_GRAD"])
-def test_c3_dana_and_sa_gradient(P, variant):
+@pytest.mark.parametrize("variant", ["DANA_GA", "DANA", "DANA_SA", "SA_GRAD", "ADAM", "ADAM_SA", "ADAM_GA"])
+def test_c3_appendix_masters(P, variant):
     """The appendix's masters on the ResNet-50 shape (64 workers), fused windows of 16."""
     import torch
     _sampled(P, "C3", variant, 16, n_arrivals=400).close()
@@ -233,6 +236,40 @@ def test_dana_push_then_pull_and_checkpoint(P):
             plain.get_worker_momentum(0)
         finally:
             plain.close()
+
+
+def test_adam_options_and_checkpoint(P):
+    """Adam-GA with non-default beta_2 / epsilon, stand-alone push + pull, export/import."""
+    import torch
+    d, n = 4099, 3
+    rng = np.random.default_rng(9)
+    th0 = rng.normal(size=d).astype(np.float32)
+    eng = P.Engine(d, n, 0.01, 0.8, 0.99, P.GA_ADAM_GA)
+    eng.set_option(P.GA_OPT_ADAM_BETA2, 0.95)
+    eng.set_option(P.GA_OPT_ADAM_EPS, 1e-6)
+    eng.set_params(torch.from_numpy(th0).cuda())
+    o = oracle.Oracle(d, n, 0.01, 0.8, 0.99, oracle.ADAM_GA, beta2=0.95, adam_eps=1e-6)
+    o.set_params(th0)
+    for i in [0, 1, 2, 1, 0, 0]:
+        g = rng.normal(size=d).astype(np.float32)
+        assert eng.push(i, torch.from_numpy(g).cuda()) == o.push(i, g)
+        assert _same(_np(eng.pull(i)), (o.pull(i), o.saved(i))[1])
+    with pytest.raises(P.GaError):
+        eng.set_option(P.GA_OPT_ADAM_BETA2, 0.9)          # not after the first arrival
+    other = P.Engine(d, n, 0.5, 0.1, 0.5, P.GA_ADAM_GA)   # hyper-parameters come with the state
+    other.import_state(eng.export_state())
+    g = rng.normal(size=d).astype(np.float32)
+    o.push_batch([2], [g])
+    for e_ in (eng, other):
+        e_.push_batch([2], [torch.from_numpy(g).cuda()])
+        for which, ref in ((P.GA_THETA, o.get(o.THETA)), (P.GA_V, o.get(o.V)), (P.GA_V2, o.second_moment()),
+                           (P.GA_M, o.get(o.M)), (P.GA_C, o.get(o.C))):
+            assert _same(_np(e_.get(which)), ref), which
+        e_.close()
+    plain = P.Engine(64, 2)
+    with pytest.raises(P.GaError):
+        plain.get(P.GA_V2)
+    plain.close()
 
 
 def test_c4_stragglers(P):
@@ -422,7 +459,7 @@ def test_bad_arguments_return_errors(P):
     assert not l.ga_create(10, 4, -1.0, 0.9, 0.999, P.GA_GA)
     assert not l.ga_create(10, 4, 0.1, 1.0, 0.999, P.GA_GA)
     assert not l.ga_create(10, 4, 0.1, 0.9, 1.0, P.GA_GA)
-    assert not l.ga_create(10, 4, 0.1, 0.9, 0.999, 7)
+    assert not l.ga_create(10, 4, 0.1, 0.9, 0.999, 10) and "variant" in P.last_error()
     assert l.ga_push(None, 0, None) == P.GA_ERR_ARG
     l.ga_destroy(None)
     eng = P.Engine(1000, 4, 0.1, -0.5, 0.999, P.GA_GA)     # negative momentum is legal
