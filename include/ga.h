@@ -99,6 +99,11 @@ void ga_destroy(ga_engine* e);
 /* Enqueue all later work of this engine on cuda_stream (a cudaStream_t; NULL = default stream). */
 int ga_set_stream(ga_engine* e, void* cuda_stream);
 
+/* Learning rate eta_k for the arrivals that follow (decay, warm-up: Appendix "Hyperparameters").
+ * eta_max of the C algorithm stays the rate given to ga_create ("usually eta_max = eta_1"), so
+ * the Gap penalty relaxes as the rate decays (Section 5.1). lr must be positive and finite. */
+int ga_set_lr(ga_engine* e, float lr);
+
 /* theta <- theta0 and every worker's saved copy <- theta0 ("Initialize theta^i = theta_0",
  * Algorithm "DANA-Gap-Aware: master" line 1; the same convention is used for GA); v, m, the
  * arrival counter and iter[] are reset to 0. theta0_dev: n_params floats on the device. */

@@ -37,6 +37,7 @@ def _bind(path):
     lib.gao_destroy.argtypes = [c.c_void_p]
     lib.gao_set_c_order.argtypes = [c.c_void_p, c.c_int]
     lib.gao_set_eps.argtypes = [c.c_void_p, c.c_double]
+    lib.gao_set_lr.argtypes = [c.c_void_p, c.c_double]
     lib.gao_set_params.argtypes = [c.c_void_p, c.c_void_p]
     lib.gao_pull.argtypes = [c.c_void_p, c.c_int]
     lib.gao_push.restype = c.c_int64
@@ -103,6 +104,9 @@ class Oracle:
         a = _f32(theta0)
         assert a.shape == (self.d,)
         self._l.gao_set_params(self._h, a.ctypes.data)
+
+    def set_lr(self, lr):
+        self._l.gao_set_lr(self._h, lr)
 
     def pull(self, worker):
         assert 0 <= worker < self.n

@@ -398,6 +398,13 @@ void gao_set_c_order(void* p, int c_order) {
     if (h->precision == 32) h->f->c_order = c_order; else h->g->c_order = c_order;
 }
 
+// Learning rate eta_k of the coming arrivals; eta_max of the C algorithm stays as created
+// (Appendix "C Coefficient": "usually eta_max = eta_1").
+void gao_set_lr(void* p, double lr) {
+    auto* h = (Handle*)p;
+    if (h->precision == 32) h->f->eta = (float)lr; else h->g->eta = (double)(float)lr;
+}
+
 void gao_set_eps(void* p, double eps) {
     auto* h = (Handle*)p;
     if (h->precision == 32) h->f->eps = (float)eps; else h->g->eps = eps;

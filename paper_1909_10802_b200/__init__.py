@@ -32,6 +32,7 @@ _SIGNATURES = {
     "ga_create": (_c.c_void_p, [_c.c_size_t, _c.c_int, _c.c_float, _c.c_float, _c.c_float, _c.c_int]),
     "ga_destroy": (None, [_c.c_void_p]),
     "ga_set_stream": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
+    "ga_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
     "ga_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
     "ga_pull": (_c.c_void_p, [_c.c_void_p, _c.c_int]),
     "ga_saved": (_c.c_void_p, [_c.c_void_p, _c.c_int]),
@@ -140,6 +141,9 @@ class Engine:
     def set_stream(self, stream):
         raw = stream if isinstance(stream, int) else stream.cuda_stream
         _check(self._l.ga_set_stream(self._h, raw))
+
+    def set_lr(self, lr):
+        _check(self._l.ga_set_lr(self._h, lr))
 
     def set_option(self, key, value):
         _check(self._l.ga_set_option(self._h, key, float(value)))
@@ -254,7 +258,7 @@ class Engine:
 
 
 # ---- checkpoint blobs (layout of ga_export_state): header, iter[N], theta, v, m, saved[N][d]
-_HEADER = "<IIqqqqffffiiiiiiff"
+_HEADER = "<IIqqqqffffiiiiiiffff"
 _MAGIC = 0x47415331
 
 
@@ -265,7 +269,7 @@ def unpack_state(blob):
     import numpy as np
     hs = struct.calcsize(_HEADER)
     (magic, version, d, n, k_done, k_c, lr, gamma, beta, eps, variant, c_order, fast_math, stats,
-     window, _, beta2, adam_eps) = struct.unpack_from(_HEADER, blob, 0)
+     window, _, beta2, adam_eps, lr_max, _) = struct.unpack_from(_HEADER, blob, 0)
     if magic != _MAGIC or version != 2:
         raise ValueError("not a Gap-Aware master checkpoint")
     off = hs
@@ -276,7 +280,7 @@ def unpack_state(blob):
     rows = 3 + n * (2 if dana else 1) + (1 if adam else 0)
     vecs = np.frombuffer(blob, dtype=np.float32, count=rows * d, offset=off).reshape(rows, d).copy()
     extra = {"v_workers": vecs[3 + n:]} if dana else {"v2": vecs[3 + n]} if adam else {}
-    extra.update(beta2=beta2, adam_eps=adam_eps)
+    extra.update(beta2=beta2, adam_eps=adam_eps, lr_max=lr_max)
     return dict(**extra, d=d, n_workers=n, k_done=k_done, k_c=k_c, lr=lr, momentum=gamma, c_beta=beta, eps=eps,
                 variant=variant, c_order=c_order, fast_math=fast_math, stats=stats, window=window,
                 iter=iters, theta=vecs[0], v=vecs[1], m=vecs[2], saved=vecs[3:3 + n])
@@ -290,7 +294,7 @@ def pack_state(st):
     head = struct.pack(_HEADER, _MAGIC, 2, st["d"], st["n_workers"], st["k_done"], st["k_c"], st["lr"],
                        st["momentum"], st["c_beta"], st["eps"], st["variant"], st["c_order"],
                        st["fast_math"], st["stats"], st["window"], 0, st.get("beta2", 0.999),
-                       st.get("adam_eps", 1e-8))
+                       st.get("adam_eps", 1e-8), st.get("lr_max", st["lr"]), 0.0)
     parts = [head, np.ascontiguousarray(st["iter"], dtype=np.int64).tobytes()]
     for name in ("theta", "v", "m", "saved") + tuple(x for x in ("v_workers", "v2") if x in st):
         a = np.ascontiguousarray(st[name], dtype=np.float32)

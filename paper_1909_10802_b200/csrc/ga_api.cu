@@ -37,7 +37,7 @@ constexpr uint32_t kStateMagic = 0x47415331;   // "GAS1"
 struct ga_engine {
     long long d = 0, stride = 0;  // parameters; padded row length in floats
     int n_workers = 0, variant = GA_GA, device = 0;
-    float lr = 0, gamma = 0, beta = 0, eps = 1e-8f;
+    float lr = 0, lr_max = 0, gamma = 0, beta = 0, eps = 1e-8f;   // lr = eta_k, lr_max = eta_max of C
     int c_order = 0, fast_math = 0, stats = 0, window = GA_MAX_WINDOW;
     float *theta = nullptr, *vel = nullptr, *mom = nullptr, *saved = nullptr;
     float* vworker = nullptr;     // DANA: N rows, v^i of every worker (vel then holds their sum)
@@ -69,7 +69,7 @@ struct ga_engine {
     bool is_tau_grad() const { return variant == GA_SA_GRAD || variant == GA_DANA_SA || variant == GA_ADAM_SA; }
     ga::Hyper hyper() const {
         ga::Hyper h;
-        h.eta_max = lr;
+        h.eta_max = lr_max;
         h.gamma = gamma;
         h.beta = beta;
         h.one_minus_beta = (float)(1.0 - (double)beta);
@@ -301,6 +301,7 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
     e->stride = (e->d + kRowAlign - 1) / kRowAlign * kRowAlign;
     e->n_workers = n_workers;
     e->lr = lr;
+    e->lr_max = lr;
     e->gamma = momentum;
     e->beta = c_beta;
     e->variant = variant;
@@ -371,6 +372,13 @@ void ga_destroy(ga_engine* e) {
 int ga_set_stream(ga_engine* e, void* cuda_stream) {
     if (int rc = check_engine(e)) return rc;
     e->stream = (cudaStream_t)cuda_stream;
+    return GA_OK;
+}
+
+int ga_set_lr(ga_engine* e, float lr) {
+    if (int rc = check_engine(e)) return rc;
+    if (!(lr > 0.f) || !std::isfinite(lr)) return fail(GA_ERR_ARG, "lr must be positive and finite");
+    e->lr = lr;
     return GA_OK;
 }
 
@@ -615,7 +623,7 @@ struct StateHeader {
     int64_t d, n_workers, k_done, k_c;
     float lr, gamma, beta, eps;
     int32_t variant, c_order, fast_math, stats, window, reserved;
-    float beta2, adam_eps;
+    float beta2, adam_eps, lr_max, pad;
 };
 
 size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
@@ -627,7 +635,7 @@ size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
     DeviceGuard guard(e->device);
     StateHeader h{};
     h.magic = kStateMagic; h.version = 2;
-    h.beta2 = e->beta2; h.adam_eps = e->adam_eps;
+    h.beta2 = e->beta2; h.adam_eps = e->adam_eps; h.lr_max = e->lr_max;
     h.d = e->d; h.n_workers = e->n_workers; h.k_done = e->k_done; h.k_c = e->k_c;
     h.lr = e->lr; h.gamma = e->gamma; h.beta = e->beta; h.eps = e->eps;
     h.variant = e->variant; h.c_order = e->c_order; h.fast_math = e->fast_math; h.stats = e->stats; h.window = e->window;
@@ -679,7 +687,7 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
     e->iter = iter;
     e->k_done = h.k_done; e->k_c = h.k_c;
     e->lr = h.lr; e->gamma = h.gamma; e->beta = h.beta; e->eps = h.eps;
-    e->beta2 = h.beta2; e->adam_eps = h.adam_eps;
+    e->beta2 = h.beta2; e->adam_eps = h.adam_eps; e->lr_max = h.lr_max;
     e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window;
     e->stats_valid = false;
     return GA_OK;

@@ -774,6 +774,49 @@ def pin_adam_exact_brute_force(make):
                     assert np.all(np.abs(got - want) <= tol * (1 + np.abs(want))), (variant, c_order, prec)
 
 
+def pin_learning_rate_schedule(make):
+    """Section 5.1: the staleness penalty should shrink as eta decays, so C keeps the MAXIMAL
+    rate (C = eta_max E|grad|) while the step uses eta_k. After the rate is cut by 10 the
+    coefficient is unchanged, the same displacement counts as the same Gap, and steps are 10x
+    shorter; for Adam and DANA the new rate enters the step / the estimate the same way."""
+    d, eta = 14, 0.1
+    r = _rng(41)
+    th0 = _f32(r.normal(size=d))
+    g = [_f32(r.normal(size=d)) for _ in range(4)]
+    o = make(d, 2, eta, 0.0, 0.999, GA, precision=64)
+    o.set_params(th0)
+    o.push(0, g[0]); o.pull(0)
+    C_before = o.get(C)
+    o.set_lr(eta / 10)
+    assert np.array_equal(o.get(C), C_before)
+    th_before, G = o.get(THETA), o.gap(1)
+    o.push(1, g[1])
+    e10 = float(np.float32(eta / 10))
+    assert np.allclose(th_before - o.get(THETA), e10 * g[1].astype(np.float64) / G, rtol=1e-12)
+    # SA: eta_k / tau
+    o = make(d, 2, eta, 0.0, 0.999, SA, precision=64)
+    o.set_params(th0)
+    o.push(0, g[0]); o.pull(0)
+    o.set_lr(eta / 10)
+    th_before = o.get(THETA)
+    assert o.push(1, g[1]) == 2
+    assert np.allclose(th_before - o.get(THETA), e10 / 2 * g[1].astype(np.float64), rtol=1e-12)
+    # DANA: the estimate uses the current rate
+    o = make(d, 1, eta, 0.5, 0.999, DANA, precision=64)
+    o.set_params(th0)
+    o.push(0, g[0])
+    o.set_lr(eta / 10)
+    o.pull(0)
+    assert np.allclose(o.saved(0), o.get(THETA) - e10 * 0.5 * g[0].astype(np.float64), rtol=1e-13)
+    # Adam: first step at the new rate
+    o = make(d, 1, eta, 0.9, 0.999, ADAM, precision=64)
+    o.set_params(th0)
+    o.set_lr(eta / 10)
+    o.push(0, g[0])
+    g64 = g[0].astype(np.float64)
+    assert np.allclose(th0.astype(np.float64) - o.get(THETA), e10 * g64 / (np.abs(g64) + 1e-8), rtol=1e-6)
+
+
 ALL_PINS = [
     pin_gap_is_one_where_copy_equals_master,
     pin_one_worker_is_heavy_ball,
@@ -796,4 +839,5 @@ ALL_PINS = [
     pin_adam_penalty_on_first_moment_only,
     pin_adam_ga_coefficient,
     pin_adam_exact_brute_force,
+    pin_learning_rate_schedule,
 ]

@@ -272,6 +272,34 @@ def test_adam_options_and_checkpoint(P):
     plain.close()
 
 
+@pytest.mark.parametrize("variant", ["GA", "SA", "DANA_GA", "ADAM_GA"])
+def test_learning_rate_schedule(P, variant):
+    """ga_set_lr between windows (a warm-up then a decay): eta_k changes, eta_max does not."""
+    import torch
+    wl = W.config("mini")
+    from paper_1909_10802_b200.runner import Run
+    run = Run(wl, variant, 4)
+    o = oracle.Oracle(wl.d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, oracle.VARIANTS[variant])
+    o.set_params(wl.theta0())
+    sched = wl.schedule()
+    k = 0
+    for lr, upto in ((wl.lr / wl.n_workers, 12), (wl.lr, 36), (wl.lr * 0.1, 60)):
+        run.engine.set_lr(lr)
+        o.set_lr(lr)
+        run.run(upto)
+        while k < upto:
+            i = sched[k]
+            o.push(i, wl.grad(k + 1, o.sent_f32(i)))
+            o.pull(i)
+            k += 1
+    _compare_engine(P, run, o, label=f"{variant} with schedule: ")
+    blob = run.engine.export_state()
+    assert abs(P.unpack_state(blob)["lr_max"] - np.float32(wl.lr)) < 1e-9
+    assert abs(P.unpack_state(blob)["lr"] - np.float32(wl.lr * 0.1)) < 1e-9
+    assert run.engine._l.ga_set_lr(run.engine._h, -1.0) == P.GA_ERR_ARG
+    run.close()
+
+
 def test_c4_stragglers(P):
     import torch
     _sampled(P, "C4", "GA", 16).close()

@@ -128,3 +128,23 @@ def test_windows_never_repeat_a_worker():
         assert [i for w in ws for i in w] == s
         assert all(len(w) <= k_max and len(set(w)) == len(w) for w in ws)
     assert W.windows([0, 1, 0, 0, 2], 16) == [[0, 1], [0], [0, 2]]
+
+
+def test_gamma_execution_time_model_matches_the_papers_figures():
+    """Appendix "Gamma Distribution": both settings have mean 128; an iteration takes at least
+    1.25x the mean with probability 1% (homogeneous) and 27.9% (heterogeneous)."""
+    homo = np.concatenate([W.gamma_task_times(s, 64, 2000).ravel() / W.gamma_task_times(s, 64, 2000).mean()
+                           for s in range(20)])
+    assert abs((homo >= 1.25).mean() - 0.01) < 0.003
+    het = np.concatenate([W.gamma_task_times(s, 512, 200, heterogeneous=True).ravel() for s in range(20)])
+    assert abs(het.mean() / 128 - 1) < 0.03
+    assert abs((het >= 160).mean() - 0.279) < 0.015
+    t = W.gamma_task_times(3, 16, 50000)
+    assert abs(t.std() / t.mean() - 0.1) < 0.005            # V_mach = 0.1
+    # heterogeneous machines keep their own mean for the whole run; homogeneous ones do not
+    th = W.gamma_task_times(4, 32, 4000, heterogeneous=True)
+    assert th.mean(axis=1).std() / th.mean() > 0.3 and t.mean(axis=1).std() / t.mean() < 0.01
+    s1 = W.schedule_gamma(5, 8, 500)
+    assert len(s1) == 500 and set(s1) == set(range(8)) and s1 == W.schedule_gamma(5, 8, 500)
+    counts = np.bincount(W.schedule_gamma(5, 16, 4000, heterogeneous=True), minlength=16)
+    assert counts.max() / max(1, counts.min()) > 2

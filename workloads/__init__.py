@@ -116,7 +116,10 @@ def _simulate(n_workers, arrivals, draw):
     for _ in range(arrivals):
         t, i = heapq.heappop(heap)
         out.append(i)
-        heapq.heappush(heap, (t + draw(i, count[i]), i))
+        nxt = draw(i, count[i])
+        if nxt is None:          # the caller's table of task times ran out
+            return None
+        heapq.heappush(heap, (t + nxt, i))
         count[i] += 1
     return out
 
@@ -149,6 +152,34 @@ def schedule_exponential_stragglers(seed, n_workers, arrivals, frac=0.1, slow=5.
     keys = [key(seed, TIME, i) for i in range(n_workers)]
     return _simulate(n_workers, arrivals,
                      lambda i, n: -scale[i] * math.log(1.0 - unit_double(word(keys[i], n))))
+
+
+def gamma_task_times(seed, n_workers, tasks_per_worker, batch=128, heterogeneous=False, v_task=0.1,
+                     v_mach=None):
+    """Execution times of the paper's gamma-distributed cluster model (Appendix "Gamma
+    Distribution", Algorithms "Task execution time - homogeneous / heterogeneous machines").
+    Returns an (n_workers, tasks_per_worker) array. Mean time = `batch` simulated units (the
+    figure's 128 for B = 128; the text's mu = B*V_mach^2 contradicts its own figure).
+    V_mach = 0.1 (homogeneous) or 0.6 (heterogeneous), V_task = 0.1; alpha = 1/V^2."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    v_mach = (0.6 if heterogeneous else 0.1) if v_mach is None else v_mach
+    a_task, a_mach, mu = 1.0 / v_task ** 2, 1.0 / v_mach ** 2, float(batch)
+    if heterogeneous:
+        p = rng.gamma(a_mach, mu / a_mach, size=n_workers)             # mean time of each machine
+        return rng.gamma(a_task, p[:, None] / a_task, size=(n_workers, tasks_per_worker))
+    q = rng.gamma(a_task, mu / a_task)                                  # drawn once
+    return rng.gamma(a_mach, q / a_mach, size=(n_workers, tasks_per_worker))
+
+
+def schedule_gamma(seed, n_workers, arrivals, heterogeneous=False, batch=128):
+    """Arrival order under the gamma execution-time model."""
+    per = arrivals // n_workers + 8
+    while True:
+        t = gamma_task_times(seed, n_workers, per, batch, heterogeneous)
+        sched = _simulate(n_workers, arrivals, lambda i, n: float(t[i, n]) if n < per else None)
+        if sched is not None:
+            return sched
+        per *= 2
 
 
 def schedule_round_robin(n_workers, arrivals):
@@ -251,7 +282,7 @@ class Workload:
     segments: list
     n_workers: int
     arrivals: int
-    schedule_kind: str            # "ticks" | "lognormal" | "exp_stragglers" | "round_robin"
+    schedule_kind: str            # "ticks" | "lognormal" | "exp_stragglers" | "round_robin" | "gamma" | "gamma_hetero"
     seed: int
     lr: float = 0.1
     momentum: float = 0.9
@@ -298,6 +329,8 @@ class Workload:
             return schedule_exponential_stragglers(self.seed, n, a)
         if kind == "round_robin":
             return schedule_round_robin(n, a)
+        if kind in ("gamma", "gamma_hetero"):
+            return schedule_gamma(self.seed, n, a, heterogeneous=(kind == "gamma_hetero"))
         raise ValueError(kind)
 
     def sample_indices(self, n, extra_seed=0):
