@@ -13,9 +13,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ga_oracle.cpp")
 _LIB = os.path.join(_HERE, "libga_oracle.so")
 
-ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA, ADAM, ADAM_SA, ADAM_GA = range(10)
+ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA, ADAM, ADAM_SA, ADAM_GA, GA_LAYER = range(11)
 VARIANTS = {"ASGD": ASGD, "SA": SA, "GA": GA, "SA_GRAD": SA_GRAD, "DANA": DANA, "DANA_SA": DANA_SA,
-            "DANA_GA": DANA_GA, "ADAM": ADAM, "ADAM_SA": ADAM_SA, "ADAM_GA": ADAM_GA}
+            "DANA_GA": DANA_GA, "ADAM": ADAM, "ADAM_SA": ADAM_SA, "ADAM_GA": ADAM_GA, "GA_LAYER": GA_LAYER}
 CXXFLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-Wall", "-Wextra"]
 
 
@@ -49,6 +49,9 @@ def _bind(path):
     lib.gao_iter.argtypes = [c.c_void_p, c.c_int]
     lib.gao_set_state.argtypes = [c.c_void_p] * 6 + [c.c_int64, c.c_int64, c.c_void_p]
     lib.gao_set_dana_sum.argtypes = [c.c_void_p, c.c_int]
+    lib.gao_set_layers.restype = c.c_int
+    lib.gao_set_layers.argtypes = [c.c_void_p, c.c_void_p, c.c_int]
+    lib.gao_layer_state.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
     lib.gao_set_adam.argtypes = [c.c_void_p, c.c_double, c.c_double]
     lib.gao_k_c.restype = c.c_int64
     lib.gao_k_c.argtypes = [c.c_void_p]
@@ -104,6 +107,19 @@ class Oracle:
         a = _f32(theta0)
         assert a.shape == (self.d,)
         self._l.gao_set_params(self._h, a.ctypes.data)
+
+    def set_layers(self, offsets):
+        """GA_LAYER: layer p = elements [offsets[p], offsets[p+1]); default is one layer (global Gap)."""
+        off = np.ascontiguousarray(offsets, dtype=np.int64)
+        assert self._l.gao_set_layers(self._h, off.ctypes.data, len(off) - 1) == 0, "bad layer offsets"
+        self.n_layers = len(off) - 1
+
+    def layer_state(self):
+        """(Gap of every layer at the last arrival, m_p of every layer)."""
+        n = getattr(self, "n_layers", 1)
+        g, m = np.empty(n), np.empty(n)
+        self._l.gao_layer_state(self._h, g.ctypes.data, m.ctypes.data)
+        return g, m
 
     def set_lr(self, lr):
         self._l.gao_set_lr(self._h, lr)

@@ -19,6 +19,9 @@
 //   push, ADAM*        : Algorithms "Adam: master", "Adam-Staleness-Aware: master" and
 //                        "Adam-Gap-Aware: master" (appendix): the penalty (1/tau or 1/G) enters
 //                        the first moment only
+//   push, GA_LAYER     : Section 5.3, the layer-wise Gap G_p = ||theta_p - theta^i_p|| / C_p + 1
+//                        (one layer = the global Gap of Definition 1); the gradient of layer
+//                        p is multiplied by 1/G_p, then the momentum step of "Gap-Aware: master"
 //   momentum           : Section 3, the variant without dampening: v <- gamma v + g
 //   push, SA_GRAD      : Algorithm "Staleness-Aware-Gradient: master" (appendix): g / tau
 //   push/pull, DANA*   : Algorithms "DANA: master", "DANA-Staleness-Aware: master" and
@@ -51,6 +54,10 @@
 //     v); c_order decides as before whether the Gap sees m before or after this arrival's refresh.
 //   * Adam's bias corrections use k = the arrival index; m_hat = m * (1/(1-beta1^k)) with the
 //     reciprocal formed in double and rounded once, as for C.
+//   * Layer-wise / global C: the C algorithm "executed per layer": m_p is the running average
+//     of the squared NORM of layer p's update vector, C_p = eta_max (sqrt(m_p / (1 - beta^k))
+//     + eps). Squared norms are accumulated in fp64 and rounded once to the working precision
+//     (a sum of millions of fp32 terms has no meaningful fp32 order). Lagged order only.
 //   * Arithmetic: every line below is one IEEE operation per symbol, in the order
 //     written, with v <- gamma*v + g_hat and theta <- theta - eta*v each a single fused
 //     multiply-add. Build with -ffp-contract=off so nothing else is fused.
@@ -72,7 +79,7 @@
 namespace {
 
 enum Variant { ASGD = 0, SA = 1, GA = 2, SA_GRAD = 3, DANA = 4, DANA_SA = 5, DANA_GA = 6,
-               ADAM = 7, ADAM_SA = 8, ADAM_GA = 9 };
+               ADAM = 7, ADAM_SA = 8, ADAM_GA = 9, GA_LAYER = 10 };
 
 template <typename T>
 struct Master {
@@ -90,6 +97,9 @@ struct Master {
     std::vector<T> vw;          // DANA: N x d, row i = v^i, worker i's momentum
     std::vector<T> vsum;        // DANA: sum_j v^j
     int dana_sum = 1;           // 1 running sum, 0 summed afresh at every send
+    std::vector<int64_t> layer_off;   // GA_LAYER: layer p = elements [layer_off[p], layer_off[p+1])
+    std::vector<T> m_layer;           // GA_LAYER: m_p of the C algorithm, one scalar per layer
+    std::vector<double> last_layer_gap;
     std::vector<T> v2;          // Adam: second moment (the first moment lives in v; gamma is beta_1)
     T beta2 = (T)0.999f;        // Adam: beta_2
     T adam_eps = (T)1e-8f;      // Adam: epsilon
@@ -120,12 +130,49 @@ struct Master {
         k_done = 0;
         k_c = 0;
         std::fill(v2.begin(), v2.end(), (T)0);
+        std::fill(m_layer.begin(), m_layer.end(), (T)0);
         std::fill(vw.begin(), vw.end(), (T)0);
         std::fill(vsum.begin(), vsum.end(), (T)0);
     }
 
     bool is_dana() const { return variant == DANA || variant == DANA_SA || variant == DANA_GA; }
     bool has_gap() const { return variant == GA || variant == DANA_GA || variant == ADAM_GA; }
+    // One arrival with the layer-wise Gap.
+    void push_layers(int i, const float* grad) {
+        const T* s = &saved[(size_t)i * d];
+        const T one_minus_beta = (T)(1.0 - (double)beta);
+        const T ib = k_c > 0 ? inv_bias() : (T)0;
+        const size_t P = m_layer.size();
+        for (size_t p = 0; p < P; ++p) {
+            const int64_t lo = layer_off[p], hi = layer_off[p + 1];
+            double dist2 = 0.0;                                   // ||theta_p - theta^i_p||^2
+            for (int64_t j = lo; j < hi; ++j) {
+                const T diff = theta[j] - s[j];
+                dist2 += (double)diff * (double)diff;
+            }
+            const T dist = (T)std::sqrt(dist2);
+            const T C = coeff(m_layer[p], ib);
+            const T G = dist / C + (T)1;
+            const T inv_gap = (T)1 / G;
+            last_layer_gap[p] = (double)G;
+            double norm2 = 0.0;                                   // ||v_{k+1,p}||^2
+            for (int64_t j = lo; j < hi; ++j) {
+                const T g_hat = inv_gap * (T)grad[j];
+                v[j] = std::fma(gamma, v[j], g_hat);
+                theta[j] = std::fma(-eta, v[j], theta[j]);
+                norm2 += (double)v[j] * (double)v[j];
+            }
+            m_layer[p] = std::fma(beta, m_layer[p], one_minus_beta * (T)norm2);
+        }
+        k_c += 1;
+    }
+
+    void set_layers(const int64_t* off, int n) {
+        layer_off.assign(off, off + n + 1);
+        m_layer.assign(n, 0);
+        last_layer_gap.assign(n, 1.0);
+    }
+
     bool is_adam() const { return variant == ADAM || variant == ADAM_SA || variant == ADAM_GA; }
 
     // One arrival of the three Adam masters. v holds the first moment, gamma is beta_1.
@@ -249,6 +296,8 @@ struct Master {
             push_dana(i, grad, tau);
         } else if (is_adam()) {
             push_adam(i, grad, k, tau);
+        } else if (variant == GA_LAYER) {
+            push_layers(i, grad);
         } else if (variant == SA_GRAD) {
             for (int64_t j = 0; j < d; ++j) {
                 const T g_tau = (T)grad[j] / (T)tau;
@@ -356,6 +405,7 @@ Master<T>* make(int64_t d, int n, double lr, double momentum, double beta, int v
     M->saved.assign((size_t)n * d, 0);
     M->iter.assign(n, 0);
     if (M->is_adam()) M->v2.assign(d, 0);
+    if (variant == GA_LAYER) { const int64_t whole[2] = {0, d}; M->set_layers(whole, 1); }
     if (M->is_dana()) {
         M->vw.assign((size_t)n * d, 0);
         M->vsum.assign(d, 0);
@@ -372,7 +422,7 @@ extern "C" {
 void* gao_create(int64_t d, int n_workers, double lr, double momentum, double beta, int variant,
                  int precision) {
     if (d <= 0 || n_workers <= 0 || (precision != 32 && precision != 64)) return nullptr;
-    if (variant < 0 || variant > 9) return nullptr;
+    if (variant < 0 || variant > 10) return nullptr;
     auto* h = new (std::nothrow) Handle{precision, nullptr, nullptr};
     if (!h) return nullptr;
     try {
@@ -421,6 +471,23 @@ void gao_set_state(void* p, const double* th, const double* v, const double* m, 
                    const int64_t* iter, int64_t k_done, int64_t k_c, const double* v_workers) {
     auto* h = (Handle*)p;
     DISPATCH(h, set_state(th, v, m, saved, iter, k_done, k_c, v_workers));
+}
+// Layers of the layer-wise Gap: offsets[0] = 0 < ... < offsets[n] = d. Resets m_p.
+int gao_set_layers(void* p, const int64_t* offsets, int n) {
+    auto* h = (Handle*)p;
+    const int64_t d = h->precision == 32 ? h->f->d : h->g->d;
+    if (n < 1 || offsets[0] != 0 || offsets[n] != d) return -1;
+    for (int q = 0; q < n; ++q) if (offsets[q + 1] <= offsets[q]) return -1;
+    DISPATCH(h, set_layers(offsets, n));
+    return 0;
+}
+// Gap and m_p of every layer at the last arrival.
+void gao_layer_state(void* p, double* gaps, double* m_layer) {
+    auto* h = (Handle*)p;
+    auto copy = [&](auto* M) {
+        for (size_t q = 0; q < M->m_layer.size(); ++q) { gaps[q] = M->last_layer_gap[q]; m_layer[q] = (double)M->m_layer[q]; }
+    };
+    if (h->precision == 32) copy(h->f); else copy(h->g);
 }
 void gao_set_adam(void* p, double beta2, double adam_eps) {
     auto* h = (Handle*)p;

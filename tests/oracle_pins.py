@@ -11,7 +11,7 @@ from fractions import Fraction
 
 import numpy as np
 
-ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA, ADAM, ADAM_SA, ADAM_GA = range(10)
+ASGD, SA, GA, SA_GRAD, DANA, DANA_SA, DANA_GA, ADAM, ADAM_SA, ADAM_GA, GA_LAYER = range(11)
 THETA, V, M, C = 0, 1, 2, 3
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
@@ -774,6 +774,133 @@ def pin_adam_exact_brute_force(make):
                     assert np.all(np.abs(got - want) <= tol * (1 + np.abs(want))), (variant, c_order, prec)
 
 
+# ------------------------------------------------------------------ layer-wise and global Gap
+def pin_layer_gap_with_one_parameter_per_layer_is_parameter_wise(make):
+    """Section 5.3: with every parameter a layer of its own the layer-wise Gap IS the
+    parameter-wise Gap (the norm of one number is its absolute value), bit for bit."""
+    d, n = 9, 3
+    r = _rng(51)
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 2, 0, 0, 2, 1]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    for prec in (32, 64):
+        a = make(d, n, 0.1, 0.9, 0.999, GA_LAYER, precision=prec)
+        a.set_layers(np.arange(d + 1))
+        b = make(d, n, 0.1, 0.9, 0.999, GA, precision=prec)
+        for o in (a, b):
+            o.set_params(th0)
+        assert a.push_batch(sched, grads) == b.push_batch(sched, grads)
+        assert np.array_equal(a.get(THETA), b.get(THETA)) and np.array_equal(a.get(V), b.get(V))
+        assert np.array_equal(a.layer_state()[1], b.get(M))
+
+
+def pin_global_gap_definition(make):
+    """Definition 1: G = ||theta_k - theta_{k-tau}|| / C + 1 with C = eta_max E||grad||: one number
+    for the whole vector. After t same-direction unpenalised steps G = t + 1 = the delay
+    (Section 5.1); the whole gradient is divided by that one number; the value follows from
+    the norms directly."""
+    d, eta, t = 6, 0.1, 5
+    c = _f32(np.linspace(0.5, 3.0, d))
+    o = make(d, 2, eta, 0.0, 0.999, GA_LAYER, precision=64)        # default: one layer = global
+    o.set_params(np.zeros(d, np.float32))
+    for _ in range(t):
+        o.push(1, c)
+        o.pull(1)
+        assert o.layer_state()[0][0] == 1.0
+    e = float(np.float32(eta))
+    c64 = c.astype(np.float64)
+    want_G = np.linalg.norm(t * e * c64) / (e * (np.linalg.norm(c64) + 1e-8)) + 1
+    assert abs(want_G - (t + 1)) < 1e-6
+    before = o.get(THETA)
+    g = _f32(np.linspace(-1, 1, d))
+    assert o.push(0, g) == t + 1
+    assert abs(o.layer_state()[0][0] - want_G) < 1e-12
+    assert np.allclose(before - o.get(THETA), e * g.astype(np.float64) / want_G, rtol=1e-12)
+    # m is the running average of the squared NORM of the update vector
+    m1 = o.layer_state()[1][0]
+    b = float(np.float32(0.999))
+    m_t = (1 - b ** t) * np.dot(c64, c64)                      # t refreshes with ||c||^2
+    want_m = b * m_t + (1 - b) * np.dot(g.astype(np.float64) / want_G, g.astype(np.float64) / want_G)
+    assert abs(m1 - want_m) <= 1e-12 * want_m
+
+
+def pin_layers_are_penalised_independently(make):
+    """Layer-wise Gap: 'every layer is penalized differently and independently'. A layer the
+    master has not moved since the worker pulled passes its gradient unpenalised (bitwise the
+    plain momentum step); a moved layer is scaled by one common factor 1/G_p."""
+    off = [0, 5, 12, 20]
+    d, eta = 20, 0.1
+    r = _rng(53)
+    th0 = _f32(r.normal(size=d))
+    g1 = _f32(r.normal(size=d))
+    g1[5:12] = 0.0                        # worker 1 leaves layer 1 alone
+    g0 = _f32(r.normal(size=d))
+    res = {}
+    for variant in (GA_LAYER, ASGD):
+        o = make(d, 2, eta, 0.9, 0.999, variant, precision=32)
+        if variant == GA_LAYER:
+            o.set_layers(off)
+        o.set_params(th0)
+        o.push(1, g1)
+        o.pull(1)
+        o.push(0, g0)
+        res[variant] = o
+    G = res[GA_LAYER].layer_state()[0]
+    assert G[1] == 1.0 and G[0] > 1.0 and G[2] > 1.0
+    assert np.array_equal(res[GA_LAYER].get(THETA)[5:12], res[ASGD].get(THETA)[5:12])
+    v_prev = g1.astype(np.float64)
+    for p, (lo, hi) in enumerate(zip(off[:-1], off[1:])):
+        ratio = (res[GA_LAYER].get(V)[lo:hi] - 0.9 * v_prev[lo:hi]) / g0.astype(np.float64)[lo:hi]
+        assert np.allclose(ratio, 1.0 / G[p], rtol=2e-5), p    # one factor per layer
+    # duplicating a layer's content leaves its Gap unchanged (both norms grow by sqrt 2)
+    a = make(10, 2, eta, 0.9, 0.999, GA_LAYER, precision=64)
+    b = make(20, 2, eta, 0.9, 0.999, GA_LAYER, precision=64)
+    h0, h1, h2 = th0[:10], g1[:10] + 1, g0[:10]
+    a.set_params(h0)
+    b.set_params(np.concatenate([h0, h0]))
+    for o, k in ((a, 1), (b, 2)):
+        o.push(1, np.concatenate([h1] * k)); o.pull(1); o.push(0, np.concatenate([h2] * k))
+    assert abs(a.layer_state()[0][0] - b.layer_state()[0][0]) < 1e-9
+    assert np.allclose(b.get(THETA)[:10], a.get(THETA), rtol=1e-9) and np.array_equal(b.get(THETA)[:10], b.get(THETA)[10:])
+
+
+def pin_layer_gap_exact_brute_force(make):
+    """Layer-wise Gap-Aware master in exact rational arithmetic (norms via exact sums)."""
+    r = _rng(54)
+    d, n, off = 5, 3, [0, 2, 5]
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 0, 2, 1, 0]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    eta, gam, beta, eps = 0.125, 0.75, 0.875, 1e-8
+    F = Fraction
+    th = [F(float(x)) for x in th0]
+    v = [F(0)] * d
+    mp = [F(0)] * (len(off) - 1)
+    saved = [list(th) for _ in range(n)]
+    refreshes = 0
+    for i, g in zip(sched, grads):
+        g = [F(float(x)) for x in g]
+        for p in range(len(off) - 1):
+            js = range(off[p], off[p + 1])
+            dist = _sqrt_fraction(sum((th[j] - saved[i][j]) ** 2 for j in js))
+            Cp = F(eta) * F(eps) if refreshes == 0 else F(eta) * (_sqrt_fraction(mp[p] / (1 - F(beta) ** refreshes)) + F(eps))
+            Gp = dist / Cp + 1
+            for j in js:
+                v[j] = F(gam) * v[j] + g[j] / Gp
+                th[j] = th[j] - F(eta) * v[j]
+            mp[p] = F(beta) * mp[p] + (1 - F(beta)) * sum(v[j] ** 2 for j in js)
+        refreshes += 1
+        saved[i] = list(th)
+    for prec, tol in ((64, 2e-13), (32, 2e-5)):
+        o = make(d, n, eta, gam, beta, GA_LAYER, precision=prec, eps=eps)
+        o.set_layers(off)
+        o.set_params(th0)
+        o.push_batch(sched, grads)
+        for got, ref in ((o.get(THETA), th), (o.get(V), v), (o.layer_state()[1], mp)):
+            want = np.array([float(x) for x in ref])
+            assert np.all(np.abs(got - want) <= tol * (1 + np.abs(want))), prec
+
+
 def pin_learning_rate_schedule(make):
     """Section 5.1: the staleness penalty should shrink as eta decays, so C keeps the MAXIMAL
     rate (C = eta_max E|grad|) while the step uses eta_k. After the rate is cut by 10 the
@@ -840,4 +967,8 @@ ALL_PINS = [
     pin_adam_ga_coefficient,
     pin_adam_exact_brute_force,
     pin_learning_rate_schedule,
+    pin_layer_gap_with_one_parameter_per_layer_is_parameter_wise,
+    pin_global_gap_definition,
+    pin_layers_are_penalised_independently,
+    pin_layer_gap_exact_brute_force,
 ]

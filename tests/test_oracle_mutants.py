@@ -93,6 +93,18 @@ MUTANTS = [
     ("adam_ga_unpenalised", "first = (one_minus_beta1 / G) * g;", "first = one_minus_beta1 * g;"),
     ("adam_ga_c_from_first_moment", "m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));\n            }\n            k_c += 1;\n        }\n        last_sum_gap",
      "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));\n            }\n            k_c += 1;\n        }\n        last_sum_gap"),
+    # layer-wise / global Gap
+    ("layer_norm_is_l1", "dist2 += (double)diff * (double)diff;", "dist2 += std::fabs((double)diff);"),
+    ("layer_norm_not_rooted", "const T dist = (T)std::sqrt(dist2);", "const T dist = (T)dist2;"),
+    ("layer_gap_without_one", "const T G = dist / C + (T)1;\n            const T inv_gap = (T)1 / G;\n            last_layer_gap",
+     "const T G = dist / C;\n            const T inv_gap = (T)1 / G;\n            last_layer_gap"),
+    ("layer_c_of_wrong_layer", "const T C = coeff(m_layer[p], ib);", "const T C = coeff(m_layer[0], ib);"),
+    ("layer_m_from_gradient", "norm2 += (double)v[j] * (double)v[j];", "norm2 += (double)grad[j] * (double)grad[j];"),
+    ("layer_m_mean_not_sum", "m_layer[p] = std::fma(beta, m_layer[p], one_minus_beta * (T)norm2);",
+     "m_layer[p] = std::fma(beta, m_layer[p], one_minus_beta * (T)(norm2 / (double)(hi - lo)));"),
+    ("layer_whole_vector_norm", "for (int64_t j = lo; j < hi; ++j) {\n                const T diff",
+     "for (int64_t j = 0; j < d; ++j) {\n                const T diff"),
+    ("layer_unpenalised", "const T g_hat = inv_gap * (T)grad[j];\n                v[j]", "const T g_hat = (T)grad[j];\n                v[j]"),
     ("dana_pull_forgets_iteration", "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);\n        }\n        iter[i] = k_done;",
      "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);\n        }"),
 ]
