@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--config", default="C5")
     ap.add_argument("--params", type=int, default=0, help="profiling aid: a one-segment vector of this size")
     ap.add_argument("--workers", type=int, default=32)
-    ap.add_argument("--variant", default="GA", choices=["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA", "ADAM", "ADAM_SA", "ADAM_GA"])
+    ap.add_argument("--variant", default="GA", choices=["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA", "ADAM", "ADAM_SA", "ADAM_GA", "GA_LAYER"])
     ap.add_argument("--window", type=int, default=16)
     ap.add_argument("--math", default="exact", choices=["exact", "fast"])
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -58,6 +58,8 @@ def parse_args():
 def bytes_per_param_window(variant, k):
     """Algorithmic bytes one parameter moves in a k-arrival window (fp32): theta, v (and m) in
     and out once; per arrival the gradient (and, for GA, the saved copy) in and the saved copy out."""
+    if variant == "GA_LAYER":                  # per arrival: norm pass 8 B, update pass 24 B; nothing fused in time
+        return 32 * k
     gap = variant in ("GA", "DANA_GA", "ADAM_GA")
     state = 24 if gap else 16                  # theta, v or sum_j v^j or Adam's m (, m behind C) in and out
     if variant.startswith("ADAM"):

@@ -56,7 +56,14 @@ enum {
      * C algorithm is run with gamma = 0, i.e. on the raw gradient, with c_beta. */
     GA_ADAM = 7,    /* m <- beta1 m + (1-beta1) g                         */
     GA_ADAM_SA = 8, /* m <- beta1 m + (1-beta1) g / tau                   */
-    GA_ADAM_GA = 9  /* m <- beta1 m + ((1-beta1)/G) g                     */
+    GA_ADAM_GA = 9, /* m <- beta1 m + ((1-beta1)/G) g                     */
+    /* Gap-Aware with the layer-wise Gap of Section 5.3: G_p = ||theta_p - theta^i_p|| / C_p + 1, one
+     * number per layer (ga_set_layers); with a single layer -- the default -- it is the global Gap
+     * of Definition 1. C_p comes from the C algorithm run on the squared norm of the layer's
+     * update vector. Norms are accumulated in fp64 and rounded to fp32 once. Each arrival takes
+     * two passes over the vector (the norm must be known before the update), so arrivals are not
+     * fused in time and ga_push_batch_host is not available for this variant. */
+    GA_GA_LAYER = 10
 };
 
 enum { GA_OK = 0, GA_ERR_ARG = -1, GA_ERR_STATE = -2, GA_ERR_OOM = -3, GA_ERR_CUDA = -4 };
@@ -103,6 +110,18 @@ int ga_set_stream(ga_engine* e, void* cuda_stream);
  * eta_max of the C algorithm stays the rate given to ga_create ("usually eta_max = eta_1"), so
  * the Gap penalty relaxes as the rate decays (Section 5.1). lr must be positive and finite. */
 int ga_set_lr(ga_engine* e, float lr);
+
+/* GA_GA_LAYER only, before the first arrival: layer p is elements [offsets_host[p],
+ * offsets_host[p+1]); n_layers + 1 increasing offsets from 0 to n_params. Resets every m_p. */
+int ga_set_layers(ga_engine* e, const int64_t* offsets_host, int n_layers);
+
+/* GA_GA_LAYER only: the number of layers in force (1 until ga_set_layers or ga_import_state says
+ * otherwise). Negative on error. */
+int ga_num_layers(ga_engine* e);
+
+/* GA_GA_LAYER only: the Gap G_p of every layer at the most recent arrival and the running second
+ * moment m_p behind C_p, n_layers floats each, into host memory (either may be NULL). */
+int ga_get_layer_state(ga_engine* e, float* gaps_host, float* m_host);
 
 /* theta <- theta0 and every worker's saved copy <- theta0 ("Initialize theta^i = theta_0",
  * Algorithm "DANA-Gap-Aware: master" line 1; the same convention is used for GA); v, m, the

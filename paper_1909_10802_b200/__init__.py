@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("GA_LIBRARY") or os.path.join(_HERE, "libga.so")   # GA_LIBRARY: another build
 
 (GA_ASGD, GA_SA, GA_GA, GA_SA_GRAD, GA_DANA, GA_DANA_SA, GA_DANA_GA, GA_ADAM, GA_ADAM_SA,
- GA_ADAM_GA) = range(10)
+ GA_ADAM_GA, GA_GA_LAYER) = range(11)
 GA_OK, GA_ERR_ARG, GA_ERR_STATE, GA_ERR_OOM, GA_ERR_CUDA = 0, -1, -2, -3, -4
 GA_THETA, GA_V, GA_M, GA_C, GA_V2 = 0, 1, 2, 3, 4
 GA_OPT_C_ORDER, GA_OPT_MATH, GA_OPT_STATS, GA_OPT_WINDOW, GA_OPT_ADAM_BETA2, GA_OPT_ADAM_EPS = range(6)
@@ -24,7 +24,7 @@ GA_MAX_WINDOW = 16
 GA_NOALLOC_MAX_PARAMS = 1 << 28
 VARIANTS = {"ASGD": GA_ASGD, "SA": GA_SA, "GA": GA_GA, "SA_GRAD": GA_SA_GRAD, "DANA": GA_DANA,
             "DANA_SA": GA_DANA_SA, "DANA_GA": GA_DANA_GA, "ADAM": GA_ADAM, "ADAM_SA": GA_ADAM_SA,
-            "ADAM_GA": GA_ADAM_GA}
+            "ADAM_GA": GA_ADAM_GA, "GA_LAYER": GA_GA_LAYER}
 
 # every symbol include/ga.h declares: name -> (restype, argtypes)
 _c = ctypes
@@ -33,6 +33,9 @@ _SIGNATURES = {
     "ga_destroy": (None, [_c.c_void_p]),
     "ga_set_stream": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
     "ga_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
+    "ga_set_layers": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_int]),
+    "ga_num_layers": (_c.c_int, [_c.c_void_p]),
+    "ga_get_layer_state": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "ga_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
     "ga_pull": (_c.c_void_p, [_c.c_void_p, _c.c_int]),
     "ga_saved": (_c.c_void_p, [_c.c_void_p, _c.c_int]),
@@ -141,6 +144,23 @@ class Engine:
     def set_stream(self, stream):
         raw = stream if isinstance(stream, int) else stream.cuda_stream
         _check(self._l.ga_set_stream(self._h, raw))
+
+    def set_layers(self, offsets):
+        import numpy as np
+        off = np.ascontiguousarray(offsets, dtype=np.int64)
+        _check(self._l.ga_set_layers(self._h, off.ctypes.data, len(off) - 1))
+
+    @property
+    def n_layers(self):
+        return _check(self._l.ga_num_layers(self._h))
+
+    def get_layer_state(self):
+        """(Gap of every layer at the last arrival, m_p of every layer) as numpy arrays."""
+        import numpy as np
+        n = self.n_layers
+        g, m = np.empty(n, np.float32), np.empty(n, np.float32)
+        _check(self._l.ga_get_layer_state(self._h, g.ctypes.data, m.ctypes.data))
+        return g, m
 
     def set_lr(self, lr):
         _check(self._l.ga_set_lr(self._h, lr))
@@ -281,6 +301,11 @@ def unpack_state(blob):
     vecs = np.frombuffer(blob, dtype=np.float32, count=rows * d, offset=off).reshape(rows, d).copy()
     extra = {"v_workers": vecs[3 + n:]} if dana else {"v2": vecs[3 + n]} if adam else {}
     extra.update(beta2=beta2, adam_eps=adam_eps, lr_max=lr_max)
+    if variant == GA_GA_LAYER:
+        at = off + 4 * rows * d
+        nl = int(np.frombuffer(blob, dtype=np.int64, count=1, offset=at)[0])
+        extra["layer_offsets"] = np.frombuffer(blob, dtype=np.int64, count=nl + 1, offset=at + 8).copy()
+        extra["m_layer"] = np.frombuffer(blob, dtype=np.float32, count=nl, offset=at + 8 * (nl + 2)).copy()
     return dict(**extra, d=d, n_workers=n, k_done=k_done, k_c=k_c, lr=lr, momentum=gamma, c_beta=beta, eps=eps,
                 variant=variant, c_order=c_order, fast_math=fast_math, stats=stats, window=window,
                 iter=iters, theta=vecs[0], v=vecs[1], m=vecs[2], saved=vecs[3:3 + n])
@@ -299,4 +324,8 @@ def pack_state(st):
     for name in ("theta", "v", "m", "saved") + tuple(x for x in ("v_workers", "v2") if x in st):
         a = np.ascontiguousarray(st[name], dtype=np.float32)
         parts.append(a.tobytes())
+    if "layer_offsets" in st:
+        lo = np.ascontiguousarray(st["layer_offsets"], dtype=np.int64)
+        parts += [np.int64(len(lo) - 1).tobytes(), lo.tobytes(),
+                  np.ascontiguousarray(st["m_layer"], dtype=np.float32).tobytes()]
     return b"".join(parts)

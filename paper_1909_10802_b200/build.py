@@ -6,7 +6,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 LIB = os.path.join(_HERE, "libga.so")
 SOURCES = [os.path.join(_HERE, "csrc", "ga_api.cu")]
-DEPENDS = SOURCES + [os.path.join(_HERE, "csrc", "ga_kernels.cuh"), os.path.join(ROOT, "include", "ga.h")]
+DEPENDS = SOURCES + [os.path.join(_HERE, "csrc", "ga_kernels.cuh"), os.path.join(_HERE, "csrc", "ga_layer_kernels.cuh"), os.path.join(ROOT, "include", "ga.h")]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include")]
 

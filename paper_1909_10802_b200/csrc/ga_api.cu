@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "ga_kernels.cuh"
+#include "ga_layer_kernels.cuh"
 
 namespace {
 
@@ -41,6 +42,15 @@ struct ga_engine {
     int c_order = 0, fast_math = 0, stats = 0, window = GA_MAX_WINDOW;
     float *theta = nullptr, *vel = nullptr, *mom = nullptr, *saved = nullptr;
     float* vworker = nullptr;     // DANA: N rows, v^i of every worker (vel then holds their sum)
+    // layer-wise Gap: layers cut into tiles, one scalar m_p / Gap / 1/Gap per layer
+    std::vector<int64_t> layer_off;
+    ga::Tile* tiles = nullptr;
+    int* tile_begin = nullptr;     // n_layers + 1
+    double* tile_partial = nullptr;
+    float *m_layer = nullptr, *layer_gap = nullptr, *layer_inv_gap = nullptr;
+    int n_tiles = 0;
+    bool is_layer() const { return variant == GA_GA_LAYER; }
+    int n_layers() const { return (int)layer_off.size() - 1; }
     float* sec = nullptr;         // Adam: second moment (vel holds the first moment, gamma is beta_1)
     float beta2 = 0.999f, adam_eps = 1e-8f;
     std::vector<int64_t> iter;
@@ -65,7 +75,7 @@ struct ga_engine {
     float* vrow(int i) const { return vworker ? vworker + (size_t)i * stride : nullptr; }
     bool is_dana() const { return variant == GA_DANA || variant == GA_DANA_SA || variant == GA_DANA_GA; }
     bool is_adam() const { return variant == GA_ADAM || variant == GA_ADAM_SA || variant == GA_ADAM_GA; }
-    bool is_gap() const { return variant == GA_GA || variant == GA_DANA_GA || variant == GA_ADAM_GA; }
+    bool is_gap() const { return variant == GA_GA || variant == GA_GA_LAYER || variant == GA_DANA_GA || variant == GA_ADAM_GA; }
     bool is_tau_grad() const { return variant == GA_SA_GRAD || variant == GA_DANA_SA || variant == GA_ADAM_SA; }
     ga::Hyper hyper() const {
         ga::Hyper h;
@@ -146,6 +156,8 @@ int grid_1d(long long n, int threads, int cap) {
 }
 
 // ----------------------------------------------------------------------------- launch
+int launch_layer_arrival(ga_engine* e, const float* grad, float* saved_row, bool write_saved, float inv_bias);
+
 template <int FAMILY, int PENALTY, bool EXACT, int C_ORDER, bool STATS>
 void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st) {
     const long long nvec = vec_end - vec_begin;
@@ -186,12 +198,78 @@ void launch_family(ga_engine* e, const ga::Window& w, long long vb, long long ve
 int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st,
                   bool allow_stats = true) {
     if (vec_end <= vec_begin || w.K <= 0) return GA_OK;
+    if (e->is_layer()) {   // a layer's norm needs the whole vector between arrivals: no fusion in time
+        if (vec_begin != 0 || vec_end != e->stride / 4)
+            return fail(GA_ERR_STATE, "the layer-wise Gap cannot run on a sub-range of the vector");
+        for (int j = 0; j < w.K; ++j)
+            if (int rc = launch_layer_arrival(e, w.grad[j], w.saved[j], w.write_saved != 0, w.inv_bias[j])) return rc;
+        return GA_OK;
+    }
     const bool stats = allow_stats && e->stats && e->is_gap();
     if (e->is_dana()) launch_family<ga::DANA>(e, w, vec_begin, vec_end, st, stats);
     else if (e->is_adam()) launch_family<ga::ADAM>(e, w, vec_begin, vec_end, st, stats);
     else launch_family<ga::MOM>(e, w, vec_begin, vec_end, st, stats);
     GA_CUDA(e, cudaGetLastError());
     if (stats) { e->stats_valid = true; e->stats_slot = w.K - 1; }
+    return GA_OK;
+}
+
+void free_layers(ga_engine* e) {
+    cudaFree(e->tiles); cudaFree(e->tile_begin); cudaFree(e->tile_partial);
+    cudaFree(e->m_layer); cudaFree(e->layer_gap); cudaFree(e->layer_inv_gap);
+    e->tiles = nullptr; e->tile_begin = nullptr; e->tile_partial = nullptr;
+    e->m_layer = e->layer_gap = e->layer_inv_gap = nullptr;
+    e->n_tiles = 0;
+}
+
+// Cut the layers into tiles and put the tables on the device. offsets: n + 1 entries.
+int build_layers(ga_engine* e, const int64_t* offsets, int n) {
+    std::vector<ga::Tile> tiles;
+    std::vector<int> begin(n + 1);
+    for (int p = 0; p < n; ++p) {
+        begin[p] = (int)tiles.size();
+        for (int64_t at = offsets[p]; at < offsets[p + 1]; at += ga::kLayerTile) {
+            ga::Tile t;
+            t.start = at;
+            t.len = (int)std::min<int64_t>(ga::kLayerTile, offsets[p + 1] - at);
+            t.layer = p;
+            tiles.push_back(t);
+        }
+    }
+    begin[n] = (int)tiles.size();
+    free_layers(e);
+    const size_t nt = tiles.size();
+    bool ok = cudaMalloc(&e->tiles, sizeof(ga::Tile) * nt) == cudaSuccess &&
+              cudaMalloc(&e->tile_begin, sizeof(int) * (n + 1)) == cudaSuccess &&
+              cudaMalloc(&e->tile_partial, sizeof(double) * nt) == cudaSuccess &&
+              cudaMalloc(&e->m_layer, sizeof(float) * n) == cudaSuccess &&
+              cudaMalloc(&e->layer_gap, sizeof(float) * n) == cudaSuccess &&
+              cudaMalloc(&e->layer_inv_gap, sizeof(float) * n) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        free_layers(e);
+        return fail(GA_ERR_OOM, "cannot allocate the layer tables");
+    }
+    GA_CUDA(e, cudaMemcpy(e->tiles, tiles.data(), sizeof(ga::Tile) * nt, cudaMemcpyHostToDevice));
+    GA_CUDA(e, cudaMemcpy(e->tile_begin, begin.data(), sizeof(int) * (n + 1), cudaMemcpyHostToDevice));
+    GA_CUDA(e, cudaMemset(e->m_layer, 0, sizeof(float) * n));
+    GA_CUDA(e, cudaMemset(e->layer_gap, 0, sizeof(float) * n));
+    e->layer_off.assign(offsets, offsets + n + 1);
+    e->n_tiles = (int)nt;
+    return GA_OK;
+}
+
+// One arrival with the layer-wise Gap: two passes over the vector and two per-layer steps.
+int launch_layer_arrival(ga_engine* e, const float* grad, float* saved_row, bool write_saved, float inv_bias) {
+    const ga::Hyper h = e->hyper();
+    const int P = e->n_layers();
+    ga::ga_layer_dist_kernel<<<e->n_tiles, ga::kLayerThreads, 0, e->stream>>>(e->theta, saved_row, e->tiles, e->tile_partial);
+    ga::ga_layer_gap_kernel<<<P, ga::kLayerThreads, 0, e->stream>>>(e->tile_partial, e->tile_begin, e->m_layer, inv_bias, h,
+                                                                    e->layer_gap, e->layer_inv_gap);
+    ga::ga_layer_update_kernel<<<e->n_tiles, ga::kLayerThreads, 0, e->stream>>>(
+        e->theta, e->vel, grad, saved_row, write_saved ? 1 : 0, e->tiles, e->layer_inv_gap, e->lr, h, e->tile_partial);
+    ga::ga_layer_refresh_kernel<<<P, ga::kLayerThreads, 0, e->stream>>>(e->tile_partial, e->tile_begin, e->m_layer, h);
+    GA_CUDA(e, cudaGetLastError());
     return GA_OK;
 }
 
@@ -294,7 +372,7 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
     if (!(lr > 0.f) || !std::isfinite(lr)) { fail(GA_ERR_ARG, "lr must be positive and finite"); return nullptr; }
     if (!(std::fabs(momentum) < 1.f)) { fail(GA_ERR_ARG, "|momentum| must be < 1"); return nullptr; }
     if (!(c_beta >= 0.f && c_beta < 1.f)) { fail(GA_ERR_ARG, "c_beta must be in [0, 1)"); return nullptr; }
-    if (variant < GA_ASGD || variant > GA_ADAM_GA) { fail(GA_ERR_ARG, "unknown variant %d", variant); return nullptr; }
+    if (variant < GA_ASGD || variant > GA_GA_LAYER) { fail(GA_ERR_ARG, "unknown variant %d", variant); return nullptr; }
     ga_engine* e = new (std::nothrow) ga_engine();
     if (!e) { fail(GA_ERR_OOM, "out of host memory"); return nullptr; }
     e->d = (long long)n_params;
@@ -341,6 +419,10 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
         ga_destroy(e);
         return nullptr;
     }
+    if (e->is_layer()) {   // until ga_set_layers says otherwise: one layer, the global Gap
+        const int64_t whole[2] = {0, e->d};
+        if (build_layers(e, whole, 1) != GA_OK) { ga_destroy(e); return nullptr; }
+    }
     return e;
 }
 
@@ -354,6 +436,7 @@ void ga_destroy(ga_engine* e) {
     cudaFree(e->saved);
     cudaFree(e->vworker);
     cudaFree(e->sec);
+    free_layers(e);
     cudaFree(e->partials);
     cudaFree(e->stats_dev);
     cudaFree(e->pull_err);
@@ -382,6 +465,37 @@ int ga_set_lr(ga_engine* e, float lr) {
     return GA_OK;
 }
 
+int ga_set_layers(ga_engine* e, const int64_t* offsets_host, int n_layers) {
+    if (int rc = check_engine(e)) return rc;
+    if (!e->is_layer()) return fail(GA_ERR_STATE, "only the GA_GA_LAYER variant has layers");
+    if (e->k_done != 0) return fail(GA_ERR_STATE, "layers can only be set before the first arrival");
+    if (!offsets_host || n_layers < 1 || n_layers > (1 << 20)) return fail(GA_ERR_ARG, "bad layer table");
+    if (offsets_host[0] != 0 || offsets_host[n_layers] != e->d)
+        return fail(GA_ERR_ARG, "layer offsets must start at 0 and end at n_params");
+    for (int p = 0; p < n_layers; ++p)
+        if (offsets_host[p + 1] <= offsets_host[p]) return fail(GA_ERR_ARG, "layer %d is empty or out of order", p);
+    DeviceGuard guard(e->device);
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    return build_layers(e, offsets_host, n_layers);
+}
+
+int ga_num_layers(ga_engine* e) {
+    if (int rc = check_engine(e)) return rc;
+    if (!e->is_layer()) return fail(GA_ERR_STATE, "only the GA_GA_LAYER variant has layers");
+    return e->n_layers();
+}
+
+int ga_get_layer_state(ga_engine* e, float* gaps_host, float* m_host) {
+    if (int rc = check_engine(e)) return rc;
+    if (!e->is_layer()) return fail(GA_ERR_STATE, "only the GA_GA_LAYER variant has layers");
+    DeviceGuard guard(e->device);
+    const size_t bytes = sizeof(float) * e->n_layers();
+    if (gaps_host) GA_CUDA(e, cudaMemcpyAsync(gaps_host, e->layer_gap, bytes, cudaMemcpyDeviceToHost, e->stream));
+    if (m_host) GA_CUDA(e, cudaMemcpyAsync(m_host, e->m_layer, bytes, cudaMemcpyDeviceToHost, e->stream));
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    return GA_OK;
+}
+
 int ga_set_params(ga_engine* e, const float* theta0_dev) {
     if (int rc = check_engine(e)) return rc;
     if (int rc = check_dev_ptr(theta0_dev, "theta0_dev")) return rc;
@@ -390,6 +504,7 @@ int ga_set_params(ga_engine* e, const float* theta0_dev) {
         theta0_dev, e->theta, e->vel, e->mom, e->saved, e->vworker, e->n_workers, e->d, e->stride);
     GA_CUDA(e, cudaGetLastError());
     if (e->sec) GA_CUDA(e, cudaMemsetAsync(e->sec, 0, sizeof(float) * (size_t)e->stride, e->stream));
+    if (e->m_layer) GA_CUDA(e, cudaMemsetAsync(e->m_layer, 0, sizeof(float) * e->n_layers(), e->stream));
     std::fill(e->iter.begin(), e->iter.end(), 0);
     e->k_done = 0;
     e->k_c = 0;
@@ -461,6 +576,7 @@ int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* cons
     if (sent_out_host)
         for (int j = 0; j < K; ++j)
             if (!sent_out_host[j]) return fail(GA_ERR_ARG, "sent_out_host[%d] is NULL", j);
+    if (e->is_layer()) return fail(GA_ERR_STATE, "the layer-wise Gap needs whole vectors on the device: use ga_push_batch");
     DeviceGuard guard(e->device);
     if (int rc = ensure_host_path(e)) return rc;
     int launches = 0;
@@ -522,6 +638,8 @@ int ga_get(ga_engine* e, int which, float* out_dev) {
     }
     if (src) {
         GA_CUDA(e, cudaMemcpyAsync(out_dev, src, sizeof(float) * (size_t)e->d, cudaMemcpyDeviceToDevice, e->stream));
+    } else if (which == GA_C && e->is_layer()) {
+        return fail(GA_ERR_STATE, "the layer-wise variant has one C per layer: see ga_get_layer_state");
     } else if (which == GA_C) {
         ga::ga_coeff_kernel<<<grid_1d(e->d, 256, 148 * 8), 256, 0, e->stream>>>(e->mom, e->inv_bias(e->k_c),
                                                                                e->hyper(), e->d, out_dev);
@@ -548,6 +666,7 @@ int ga_gap(ga_engine* e, int worker, float* gap_out_dev) {
     if (int rc = check_engine(e)) return rc;
     if (int rc = check_worker(e, worker)) return rc;
     if (int rc = check_dev_ptr(gap_out_dev, "gap_out_dev")) return rc;
+    if (e->is_layer()) return fail(GA_ERR_STATE, "the layer-wise variant has one Gap per layer: see ga_get_layer_state");
     DeviceGuard guard(e->device);
     ga::ga_gap_kernel<<<grid_1d(e->d, 256, 148 * 8), 256, 0, e->stream>>>(
         e->theta, e->row(worker), e->mom, e->inv_bias(e->k_c), e->hyper(), e->d, gap_out_dev);
@@ -562,6 +681,7 @@ int ga_set_option(ga_engine* e, int key, double value) {
     switch (key) {
         case GA_OPT_C_ORDER:
             if (v != 0 && v != 1) return fail(GA_ERR_ARG, "GA_OPT_C_ORDER must be 0 or 1");
+            if (v == 1 && e->is_layer()) return fail(GA_ERR_STATE, "the layer-wise Gap has the lagged order only");
             if (e->k_done != 0) return fail(GA_ERR_STATE, "GA_OPT_C_ORDER can only change before the first arrival");
             e->c_order = v;
             return GA_OK;
@@ -630,7 +750,8 @@ size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
     if (check_engine(e)) return 0;
     const size_t vec = sizeof(float) * (size_t)e->d;
     const size_t rows = 3 + (size_t)e->n_workers * (e->is_dana() ? 2 : 1) + (e->is_adam() ? 1 : 0);
-    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows;
+    const size_t layer_bytes = e->is_layer() ? sizeof(int64_t) * (e->n_layers() + 2) + sizeof(float) * e->n_layers() : 0;
+    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows + layer_bytes;
     if (!buf_host || cap < need) return need;
     DeviceGuard guard(e->device);
     StateHeader h{};
@@ -650,7 +771,13 @@ size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
         err = cudaMemcpyAsync(p, e->row(i), vec, cudaMemcpyDeviceToHost, e->stream);
     for (int i = 0; e->is_dana() && i < e->n_workers && err == cudaSuccess; ++i, p += vec)
         err = cudaMemcpyAsync(p, e->vrow(i), vec, cudaMemcpyDeviceToHost, e->stream);
-    if (e->is_adam() && err == cudaSuccess) err = cudaMemcpyAsync(p, e->sec, vec, cudaMemcpyDeviceToHost, e->stream);
+    if (e->is_adam() && err == cudaSuccess) { err = cudaMemcpyAsync(p, e->sec, vec, cudaMemcpyDeviceToHost, e->stream); p += vec; }
+    if (e->is_layer() && err == cudaSuccess) {   // n_layers, offsets[n+1], m_p[n]
+        const int64_t n = e->n_layers();
+        std::memcpy(p, &n, sizeof n); p += sizeof n;
+        std::memcpy(p, e->layer_off.data(), sizeof(int64_t) * (n + 1)); p += sizeof(int64_t) * (n + 1);
+        err = cudaMemcpyAsync(p, e->m_layer, sizeof(float) * n, cudaMemcpyDeviceToHost, e->stream);
+    }
     if (err == cudaSuccess) err = cudaStreamSynchronize(e->stream);
     if (err != cudaSuccess) { cuda_fail(e, err, "ga_export_state"); return 0; }
     return need;
@@ -667,8 +794,16 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
     const size_t vec = sizeof(float) * (size_t)e->d;
     if (h.variant != e->variant) return fail(GA_ERR_ARG, "state is for variant %d, engine is variant %d", h.variant, e->variant);
     const size_t rows = 3 + (size_t)e->n_workers * (e->is_dana() ? 2 : 1) + (e->is_adam() ? 1 : 0);
-    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows;
-    if (len < need) return fail(GA_ERR_ARG, "state buffer truncated");
+    const size_t layer_bytes = e->is_layer() ? sizeof(int64_t) * (e->n_layers() + 2) + sizeof(float) * e->n_layers() : 0;
+    const size_t need = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows + layer_bytes;
+    if (e->is_layer()) {   // the layer table decides the true length
+        const size_t base = sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows;
+        if (len < base + sizeof(int64_t)) return fail(GA_ERR_ARG, "state buffer truncated");
+        int64_t n = 0;
+        std::memcpy(&n, (const char*)buf_host + base, sizeof n);
+        if (n < 1 || n > (1 << 20) || len < base + sizeof(int64_t) * (n + 2) + sizeof(float) * n)
+            return fail(GA_ERR_ARG, "state buffer truncated");
+    } else if (len < need) return fail(GA_ERR_ARG, "state buffer truncated");
     if ( h.window < 1 || h.window > GA_MAX_WINDOW || h.k_done < 0 || h.k_c < 0)
         return fail(GA_ERR_ARG, "state header holds invalid values");
     DeviceGuard guard(e->device);
@@ -682,7 +817,17 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
         GA_CUDA(e, cudaMemcpyAsync(e->row(i), p, vec, cudaMemcpyHostToDevice, e->stream));
     for (int i = 0; e->is_dana() && i < e->n_workers; ++i, p += vec)
         GA_CUDA(e, cudaMemcpyAsync(e->vrow(i), p, vec, cudaMemcpyHostToDevice, e->stream));
-    if (e->is_adam()) GA_CUDA(e, cudaMemcpyAsync(e->sec, p, vec, cudaMemcpyHostToDevice, e->stream));
+    if (e->is_adam()) { GA_CUDA(e, cudaMemcpyAsync(e->sec, p, vec, cudaMemcpyHostToDevice, e->stream)); p += vec; }
+    if (e->is_layer()) {
+        int64_t n = 0;
+        std::memcpy(&n, p, sizeof n); p += sizeof n;
+        std::vector<int64_t> off(n + 1);
+        std::memcpy(off.data(), p, sizeof(int64_t) * (n + 1)); p += sizeof(int64_t) * (n + 1);
+        if (off[0] != 0 || off[n] != e->d) return fail(GA_ERR_ARG, "state holds a layer table for another vector");
+        for (int64_t q = 0; q < n; ++q) if (off[q + 1] <= off[q]) return fail(GA_ERR_ARG, "state holds a bad layer table");
+        if (int rc = build_layers(e, off.data(), (int)n)) return rc;
+        GA_CUDA(e, cudaMemcpyAsync(e->m_layer, p, sizeof(float) * n, cudaMemcpyHostToDevice, e->stream));
+    }
     GA_CUDA(e, cudaStreamSynchronize(e->stream));
     e->iter = iter;
     e->k_done = h.k_done; e->k_c = h.k_c;

@@ -22,6 +22,9 @@ class Run:
         self.window = window
         self.engine = Engine(self.n, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, VARIANTS[variant])
         self.engine.set_option(GA_OPT_WINDOW, window)
+        if variant == "GA_LAYER":          # the workload's tensors are the layers
+            assert shard is None, "a layer's norm needs the whole layer on one rank"
+            self.engine.set_layers(wl.seg_off)
         for key, value in (options or {}).items():
             self.engine.set_option(key, value)
         theta0 = torch.empty(self.n, dtype=torch.float32, device=torch_device)

@@ -13,6 +13,9 @@ def run_oracle(wl, variant, n_arrivals=None, idx=None, precision=32, c_order=0, 
     o = oracle.Oracle(d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta,
                       oracle.VARIANTS[variant],
                       precision=precision, c_order=c_order)
+    if variant == "GA_LAYER":
+        assert idx is None, "layer norms need whole layers"
+        o.set_layers(wl.seg_off)
     o.set_params(wl.theta0(idx))
     sched = (schedule if schedule is not None else wl.schedule())
     sched = sched[:n_arrivals if n_arrivals is not None else len(sched)]

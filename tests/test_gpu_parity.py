@@ -61,6 +61,11 @@ def _compare_engine(P, run, o, idx=None, label=""):
     if run.engine.variant in (P.GA_DANA, P.GA_DANA_SA, P.GA_DANA_GA):
         names += tuple((f"v^{i}", ("vw", i), None) for i in range(run.engine.n_workers))
     names += tuple((f"sent^{i}", ("sent", i), None) for i in range(min(run.engine.n_workers, 8)))
+    if run.engine.variant == P.GA_GA_LAYER:
+        gaps, m_layer = run.engine.get_layer_state()
+        ogaps, om = o.layer_state()
+        assert np.array_equal(gaps, ogaps.astype(np.float32)), f"{label}layer Gaps differ"
+        assert np.array_equal(m_layer, om.astype(np.float32)), f"{label}layer m differ"
     for name, which, owhich in names:
         if isinstance(which, tuple):
             kind, i = which
@@ -108,7 +113,8 @@ def test_device_generator_sparse_rows_and_subrange(P):
 
 
 # ----------------------------------------------------------------------------- small, exhaustive
-ALL_VARIANTS = ["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA", "ADAM", "ADAM_SA", "ADAM_GA"]
+ALL_VARIANTS = ["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA", "ADAM", "ADAM_SA", "ADAM_GA",
+                "GA_LAYER"]
 
 
 @pytest.mark.parametrize("variant", ALL_VARIANTS)
@@ -300,6 +306,79 @@ def test_learning_rate_schedule(P, variant):
     run.close()
 
 
+def test_layer_gap_shapes(P):
+    """Layer-wise Gap on real layer tables: ResNet-20 (65 tensors, some of 10 or 16 elements,
+    odd offsets at the end) for 300 arrivals and ResNet-50 (161 tensors, 25.5M parameters, tiles
+    of 4096) for 40 arrivals; the oracle runs on whole vectors."""
+    import torch
+    from paper_1909_10802_b200.runner import Run
+    c1 = W.config("C1")
+    r50 = W.Workload(name="r50x8", segments=W.resnet50_segments(), n_workers=8, arrivals=40,
+                     schedule_kind="ticks", seed=77, sigma="loguniform")
+    for wl, n in ((c1, 300), (r50, 40)):
+        run = Run(wl, "GA_LAYER", 16)
+        run.run(n)
+        o, odelays, _ = run_oracle(wl, "GA_LAYER", n_arrivals=n)
+        assert run.delays == odelays
+        _compare_engine(P, run, o, label=f"{wl.name}/layer-wise: ")
+        gaps = run.engine.get_layer_state()[0]
+        assert gaps.min() >= 1.0 and gaps.max() > 1.5
+        run.close()
+        torch.cuda.empty_cache()
+
+
+def test_layer_gap_special_cases_and_checkpoint(P):
+    """One parameter per layer equals the parameter-wise kernel bit for bit; no layer table
+    means the global Gap; the state (layer table and m_p included) survives export/import."""
+    import torch
+    d, n = 1537, 3
+    rng = np.random.default_rng(12)
+    th0 = torch.from_numpy(rng.normal(size=d).astype(np.float32)).cuda()
+    sched = [0, 1, 2, 1, 0, 2, 2]
+    grads = [torch.from_numpy(rng.normal(size=d).astype(np.float32)).cuda() for _ in sched]
+    a = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA_LAYER)
+    a.set_layers(np.arange(d + 1))
+    b = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA)
+    for e_ in (a, b):
+        e_.set_params(th0)
+    assert a.push_batch(sched, grads) == b.push_batch(sched, grads)
+    assert torch.equal(a.get(P.GA_THETA), b.get(P.GA_THETA)) and torch.equal(a.get(P.GA_V), b.get(P.GA_V))
+    assert np.array_equal(a.get_layer_state()[1], _np(b.get(P.GA_M)))
+    a.close()
+    b.close()
+    # global Gap + checkpoint
+    g = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA_LAYER)
+    o = oracle.Oracle(d, n, 0.1, 0.9, 0.999, oracle.GA_LAYER)
+    g.set_params(th0)
+    o.set_params(_np(th0))
+    g.push_batch(sched[:4], grads[:4])
+    o.push_batch(sched[:4], [_np(x) for x in grads[:4]])
+    h = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA_LAYER)
+    h.set_layers([0, 100, d])                # replaced by the table in the state
+    blob = g.export_state()
+    h.import_state(blob)
+    st = P.unpack_state(blob)
+    assert list(st["layer_offsets"]) == [0, d] and P.pack_state(st) == blob
+    o.push_batch(sched[4:], [_np(x) for x in grads[4:]])
+    for e_ in (g, h):
+        e_.push_batch(sched[4:], grads[4:])
+        assert _same(_np(e_.get(P.GA_THETA)), o.get(o.THETA))
+        assert np.array_equal(e_.get_layer_state()[0], o.layer_state()[0].astype(np.float32))
+    # what this variant does not offer comes back as an error, not a fault
+    l = P.lib()
+    assert l.ga_set_layers(g._h, None, 1) == P.GA_ERR_STATE            # after the first arrival
+    assert l.ga_gap(g._h, 0, th0.data_ptr()) == P.GA_ERR_STATE
+    assert l.ga_set_option(h._h, P.GA_OPT_C_ORDER, 1.0) == P.GA_ERR_STATE
+    plain = P.Engine(64, 2)
+    assert l.ga_set_layers(plain._h, None, 1) == P.GA_ERR_STATE
+    fresh = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA_LAYER)
+    import ctypes
+    bad = (ctypes.c_int64 * 3)(0, 50, d - 1)
+    assert l.ga_set_layers(fresh._h, bad, 2) == P.GA_ERR_ARG
+    for e_ in (g, h, plain, fresh):
+        e_.close()
+
+
 def test_c4_stragglers(P):
     import torch
     _sampled(P, "C4", "GA", 16).close()
@@ -487,7 +566,7 @@ def test_bad_arguments_return_errors(P):
     assert not l.ga_create(10, 4, -1.0, 0.9, 0.999, P.GA_GA)
     assert not l.ga_create(10, 4, 0.1, 1.0, 0.999, P.GA_GA)
     assert not l.ga_create(10, 4, 0.1, 0.9, 1.0, P.GA_GA)
-    assert not l.ga_create(10, 4, 0.1, 0.9, 0.999, 10) and "variant" in P.last_error()
+    assert not l.ga_create(10, 4, 0.1, 0.9, 0.999, 11) and "variant" in P.last_error()
     assert l.ga_push(None, 0, None) == P.GA_ERR_ARG
     l.ga_destroy(None)
     eng = P.Engine(1000, 4, 0.1, -0.5, 0.999, P.GA_GA)     # negative momentum is legal
