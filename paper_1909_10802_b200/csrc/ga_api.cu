@@ -165,10 +165,11 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
     // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner
     if (w.K == 1)
-        ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, 1><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
+        ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, 1, 0><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
             e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
-    else
-        ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, GA_WINDOW_BATCH><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
+    else   // Adam-GA is bound by its arithmetic, not by loads in flight: it keeps the register path
+        ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, GA_WINDOW_BATCH,
+                             (FAMILY == ga::ADAM && PENALTY == ga::PEN_GAP) ? 0 : GA_WINDOW_STAGES><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
             e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
     if (STATS) {
         ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev);
