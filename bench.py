@@ -32,7 +32,7 @@ UNIT = "param-updates/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the last
 # ncu capture (profiles/), keyed by (variant, window); None once the kernel changed since.
-NCU_TRAFFIC_BYTES_PER_PARAM = {}
+NCU_TRAFFIC_BYTES_PER_PARAM = {("GA", 16, "exact"): 212.7}   # profiles/ga_window_kernel_16M_k16_full.md
 
 
 def parse_args():
