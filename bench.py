@@ -32,7 +32,7 @@ UNIT = "param-updates/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the last
 # ncu capture (profiles/), keyed by (variant, window); None once the kernel changed since.
-NCU_TRAFFIC_BYTES_PER_PARAM = {("GA", 16, "exact"): 212.7}   # profiles/ga_window_kernel_16M_k16_full.md
+NCU_TRAFFIC_BYTES_PER_PARAM = {("GA", 16, "exact"): 212.6}   # profiles/ga_window_kernel_16M_k16_full.md
 
 
 def parse_args():
@@ -276,7 +276,11 @@ def run_ours(args):
     full = [(m, n) for m, (_, _, n) in zip(ms, events) if n == args.window]
     traffic_pp = NCU_TRAFFIC_BYTES_PER_PARAM.get((args.variant, args.window, args.math))
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": traffic_pp * wl.d if traffic_pp else None, "peak_source": peak_src,
+                # measured DRAM bytes of a full window, scaled to the average launch of this run
+                # (windows cut short by a repeated worker move proportionally fewer bytes)
+                "traffic": (traffic_pp * wl.d * (alg_bytes / max(1, launches)) /
+                            (bytes_per_param_window(args.variant, args.window) * wl.d)) if traffic_pp else None,
+                "peak_source": peak_src,
                 "kernel": "ga_window_kernel", "algorithmic_bytes_per_launch": alg_bytes / max(1, launches),
                 "avg_launch_ms": sum(ms) / max(1, launches),
                 "frac_of_nominal_8TBs": achieved / 8000.0,
