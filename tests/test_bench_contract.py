@@ -1,0 +1,47 @@
+"""bench.py prints one JSON line with the agreed keys (reference arm on CPU, GPU arm on a small case)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+BASE_KEYS = {"metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+             "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e", "gpu_launches"}
+
+
+def _run(*args):
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], capture_output=True, text=True,
+                         cwd=ROOT, timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    return json.loads(lines[0])
+
+
+def test_reference_arm_times_the_oracle():
+    j = _run("--impl", "reference", "--params", "200000", "--workers", "8", "--steps", "2", "--warmup", "1")
+    assert BASE_KEYS <= set(j) and j["impl"] == "reference" and j["value"] > 0
+    assert j["cpu_baseline"]["kind"] == "oracle" and j["cpu_baseline"]["cores"] == 1
+    assert j["e2e"] == {"value": j["value"], "unit": j["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert j["metric"] == "ga_master_param_updates_per_sec" and j["higher_is_better"] is True
+
+
+def test_reference_arm_other_ranks_stay_silent():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--params", "1000"],
+                         capture_output=True, text=True, cwd=ROOT, env=env, timeout=300)
+    assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+@pytest.mark.gpu
+def test_gpu_arm_small_case():
+    j = _run("--params", "300000", "--workers", "12", "--steps", "4", "--warmup", "3", "--cpu-sample-params", "100000",
+             "--e2e-steps", "1", "--e2e-window", "4")
+    assert BASE_KEYS | {"roofline", "clocks"} <= set(j)
+    assert j["n_gpus"] == 1 and j["steps"] == 4 and j["gpu_launches"] == 4 and j["dtype"] == "f32"
+    r = j["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    assert j["e2e"]["h2d_bytes_per_step"] > 0 and j["e2e"]["d2h_bytes_per_step"] > 0 and j["e2e"]["value"] > 0
+    assert j["cpu_baseline"]["value"] > 0 and "workload" in j["config"]

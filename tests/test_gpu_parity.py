@@ -379,6 +379,27 @@ def test_layer_gap_special_cases_and_checkpoint(P):
         e_.close()
 
 
+def test_sharded_runs_equal_the_whole(P):
+    """The N > 1 layout on one GPU, one shard after the other: each rank owns a 128-byte aligned
+    range of the vector; put together the shards are the single-engine result bit for bit."""
+    import torch
+    from paper_1909_10802_b200.runner import Run
+    from paper_1909_10802_b200.shard import shard_range
+    wl = W.config("mini")
+    whole = Run(wl, "DANA_GA", 16)
+    whole.run()
+    parts = []
+    for rank in range(3):
+        j0, n = shard_range(wl.d, rank, 3)
+        part = Run(wl, "DANA_GA", 16, shard=(j0, n))
+        assert part.run() == whole.delays
+        parts.append((part.engine.get(P.GA_THETA), part.engine.get(P.GA_M), part.engine.saved(1).clone()))
+        part.close()
+    for q, ref in enumerate((whole.engine.get(P.GA_THETA), whole.engine.get(P.GA_M), whole.engine.saved(1))):
+        assert torch.equal(torch.cat([p[q] for p in parts]), ref)
+    whole.close()
+
+
 def test_c4_stragglers(P):
     import torch
     _sampled(P, "C4", "GA", 16).close()
