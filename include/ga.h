@@ -80,10 +80,12 @@ enum {
                            printed line of the C algorithm), then C, Gap and the step follow. */
     GA_OPT_MATH = 1,    /* 0 (default): every operation IEEE round-to-nearest, in the order of
                            the algorithms. 1: fast: approximate reciprocal and square root, one
-                           division per element (g*C/(|theta-theta^i|+C)); a few ulp off. */
+                           division per element (g*C/(|theta-theta^i|+C)); a few ulp off. Applies
+                           to GA_GA and GA_DANA_GA; every other variant is always exact. */
     GA_OPT_STATS = 2,   /* 1: every GA push also reduces sum and max of the Gap over all
                            parameters (the quantity the paper logs per epoch, Appendix
-                           "Gap and Delay"); read with ga_get_stats. Default 0. */
+                           "Gap and Delay"); read with ga_get_stats. Default 0. Not computed by
+                           ga_push_batch_host, nor for GA_GA_LAYER (see ga_get_layer_state). */
     GA_OPT_WINDOW = 3,  /* 1..16 (default 16): most arrivals fused into one launch by
                            ga_push_batch. */
     GA_OPT_ADAM_BETA2 = 4, /* Adam variants: beta_2 in [0,1), default 0.999; before the first arrival */

@@ -610,6 +610,50 @@ def test_bad_arguments_return_errors(P):
     eng.close()
 
 
+def test_no_write_outside_the_callers_buffers(P):
+    """Canary words around every caller-owned buffer (ragged d, so the last vector is partial):
+    outputs are written for exactly n_params floats, gradients are never written at all."""
+    import torch
+    d, pad = 10_007, 64
+    canary = 12345.0
+
+    def guarded():
+        t = torch.full((d + 2 * pad,), canary, device="cuda")
+        return t, t[pad:pad + d]
+
+    def intact(t):
+        return bool((t[:pad] == canary).all() and (t[pad + d:] == canary).all())
+
+    for variant in (P.GA_GA, P.GA_DANA_GA, P.GA_ADAM_GA, P.GA_GA_LAYER):
+        eng = P.Engine(d, 3, 0.1, 0.9, 0.999, variant)
+        full0, th0 = guarded()
+        th0.normal_()
+        eng.set_params(th0)
+        grads = [guarded() for _ in range(3)]
+        for _, g in grads:
+            g.normal_()
+        before = [full.clone() for full, _ in grads]
+        eng.push_batch([0, 1, 2], [g for _, g in grads])
+        eng.push(1, grads[0][1])
+        eng.pull(1)
+        assert all(torch.equal(full, b) for (full, _), b in zip(grads, before)) and intact(full0)
+        outs = []
+        for which in (P.GA_THETA, P.GA_V, P.GA_M) + ((P.GA_C,) if variant != P.GA_GA_LAYER else ()):
+            full, view = guarded()
+            eng.get(which, view)
+            outs.append(full)
+        if variant != P.GA_GA_LAYER:
+            full, view = guarded()
+            eng.gap(2, view)
+            outs.append(full)
+        if variant == P.GA_DANA_GA:
+            full, view = guarded()
+            eng.get_worker_momentum(0, view)
+            outs.append(full)
+        assert all(intact(o) for o in outs)
+        eng.close()
+
+
 def test_non_finite_gradient_propagates(P):
     import torch
     eng, o, rng = _small_engine(P, d=257, n=2)
