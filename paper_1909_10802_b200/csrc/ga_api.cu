@@ -526,7 +526,8 @@ const float* ga_pull(ga_engine* e, int worker) {
     }
     const long long bytes = e->stride * (long long)sizeof(float);
     const long long chunks = (bytes + ga::kPullChunk - 1) / ga::kPullChunk;
-    const int grid = (int)(chunks < 148 * 3 ? chunks : 148 * 3);
+    const long long max_grid = (long long)(e->stats_blocks / 8) * ga::kPullBlocksPerSm;   // SMs x blocks per SM
+    const int grid = (int)(chunks < max_grid ? chunks : max_grid);
     ga::ga_pull_bulk_kernel<<<grid, 32, ga::kPullStages * ga::kPullChunk, e->stream>>>(
         e->theta, e->row(worker), bytes, e->pull_err);
     cudaError_t err = cudaGetLastError();
