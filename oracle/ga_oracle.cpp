@@ -101,12 +101,20 @@ struct Master {
     std::vector<T> m_layer;           // GA_LAYER: m_p of the C algorithm, one scalar per layer
     std::vector<double> last_layer_gap;
     std::vector<T> v2;          // Adam: second moment (the first moment lives in v; gamma is beta_1)
+    T wd = 0;                   // weight decay lambda
     T beta2 = (T)0.999f;        // Adam: beta_2
     T adam_eps = (T)1e-8f;      // Adam: epsilon
     std::vector<int64_t> iter;  // iteration array of the SA algorithm
     int64_t k_done = 0;         // arrivals applied so far
     int64_t k_c = 0;            // refreshes of m so far
     double last_sum_gap = 0.0, last_max_gap = 0.0;
+
+    // The gradient the master works with. Appendix "Weight Decay": under GA the gradient
+    // contains the weight-decay element, which is divided by the Gap as a part of the gradient;
+    // the master forms it from its current parameters, g + lambda * theta_k (one FMA).
+    T gw(const float* grad, int64_t j) const {
+        return wd == (T)0 ? (T)grad[j] : std::fma(wd, theta[j], (T)grad[j]);
+    }
 
     // 1 / (1 - beta^k) of the bias correction, k = refreshes of m so far (k >= 1).
     T inv_bias() const { return (T)(1.0 / (1.0 - std::pow((double)beta, (double)k_c))); }
@@ -157,7 +165,7 @@ struct Master {
             last_layer_gap[p] = (double)G;
             double norm2 = 0.0;                                   // ||v_{k+1,p}||^2
             for (int64_t j = lo; j < hi; ++j) {
-                const T g_hat = inv_gap * (T)grad[j];
+                const T g_hat = inv_gap * gw(grad, j);
                 v[j] = std::fma(gamma, v[j], g_hat);
                 theta[j] = std::fma(-eta, v[j], theta[j]);
                 norm2 += (double)v[j] * (double)v[j];
@@ -187,14 +195,14 @@ struct Master {
         double sum_gap = 0.0, max_gap = 0.0;
         if (variant == ADAM_GA && c_order == 1) {
             for (int64_t j = 0; j < d; ++j) {
-                const T g = (T)grad[j];
+                const T g = gw(grad, j);
                 m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));
             }
             k_c += 1;
         }
         const T ib = k_c > 0 ? inv_bias() : (T)0;
         for (int64_t j = 0; j < d; ++j) {
-            const T g = (T)grad[j];
+            const T g = gw(grad, j);
             T first;                                         // what is added to beta_1 m
             if (variant == ADAM) {
                 first = one_minus_beta1 * g;
@@ -213,14 +221,10 @@ struct Master {
             const T m_hat = v[j] * inv_bias1;
             const T v_hat = v2[j] * inv_bias2;
             theta[j] = theta[j] - (eta * m_hat) / (std::sqrt(v_hat) + adam_eps);
-        }
-        if (variant == ADAM_GA && c_order == 0) {
-            for (int64_t j = 0; j < d; ++j) {
-                const T g = (T)grad[j];
+            if (variant == ADAM_GA && c_order == 0)          // lagged: C's state sees g after the Gap used it
                 m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));
-            }
-            k_c += 1;
         }
+        if (variant == ADAM_GA && c_order == 0) k_c += 1;
         last_sum_gap = sum_gap;
         last_max_gap = max_gap;
     }
@@ -253,14 +257,14 @@ struct Master {
         double sum_gap = 0.0, max_gap = 0.0;
         if (variant == DANA_GA && c_order == 1) {
             for (int64_t j = 0; j < d; ++j) {
-                const T u = std::fma(gamma, vi[j], (T)grad[j]);
+                const T u = std::fma(gamma, vi[j], gw(grad, j));
                 m[j] = std::fma(beta, m[j], one_minus_beta * (u * u));
             }
             k_c += 1;
         }
         const T ib = k_c > 0 ? inv_bias() : (T)0;
         for (int64_t j = 0; j < d; ++j) {
-            const T g = (T)grad[j];
+            const T g = gw(grad, j);
             T g_pen = g;                                   // DANA: the gradient as it is
             if (variant == DANA_SA) {
                 g_pen = g / (T)tau;                        // DANA-SA: g / tau
@@ -300,20 +304,20 @@ struct Master {
             push_layers(i, grad);
         } else if (variant == SA_GRAD) {
             for (int64_t j = 0; j < d; ++j) {
-                const T g_tau = (T)grad[j] / (T)tau;
+                const T g_tau = gw(grad, j) / (T)tau;
                 v[j] = std::fma(gamma, v[j], g_tau);
                 theta[j] = std::fma(-eta, v[j], theta[j]);
             }
         } else if (variant == ASGD) {
             for (int64_t j = 0; j < d; ++j) {
-                const T g = (T)grad[j];
+                const T g = gw(grad, j);
                 v[j] = std::fma(gamma, v[j], g);
                 theta[j] = std::fma(-eta, v[j], theta[j]);
             }
         } else if (variant == SA) {
             const T eta_tau = eta / (T)tau;
             for (int64_t j = 0; j < d; ++j) {
-                const T g = (T)grad[j];
+                const T g = gw(grad, j);
                 v[j] = std::fma(gamma, v[j], g);
                 theta[j] = std::fma(-eta_tau, v[j], theta[j]);
             }
@@ -323,14 +327,14 @@ struct Master {
             if (c_order == 1) {
                 // Adam order: refresh m from u = gamma v + g (raw gradient) first.
                 for (int64_t j = 0; j < d; ++j) {
-                    const T u = std::fma(gamma, v[j], (T)grad[j]);
+                    const T u = std::fma(gamma, v[j], gw(grad, j));
                     m[j] = std::fma(beta, m[j], one_minus_beta * (u * u));
                 }
                 k_c += 1;
             }
             const T ib = k_c > 0 ? inv_bias() : (T)0;
             for (int64_t j = 0; j < d; ++j) {
-                const T g = (T)grad[j];
+                const T g = gw(grad, j);
                 const T C = coeff(m[j], ib);
                 const T dist = std::fabs(theta[j] - s[j]);
                 const T G = dist / C + (T)1;
@@ -453,6 +457,11 @@ void gao_set_c_order(void* p, int c_order) {
 void gao_set_lr(void* p, double lr) {
     auto* h = (Handle*)p;
     if (h->precision == 32) h->f->eta = (float)lr; else h->g->eta = (double)(float)lr;
+}
+
+void gao_set_weight_decay(void* p, double wd) {
+    auto* h = (Handle*)p;
+    if (h->precision == 32) h->f->wd = (float)wd; else h->g->wd = (double)(float)wd;
 }
 
 void gao_set_eps(void* p, double eps) {

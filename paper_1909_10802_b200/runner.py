@@ -32,6 +32,8 @@ class Run:
         self.engine.set_params(theta0)
         del theta0
         self.grads = [torch.empty(self.n, dtype=torch.float32, device=torch_device) for _ in range(window)]
+        self._rows = [self.engine.saved_ptr(i) for i in range(wl.n_workers)]   # stable for the engine's life
+        self._grad_ptrs = [g.data_ptr() for g in self.grads]
         self.k = 0            # arrivals applied
         self.delays = []
         self.launches = 0
@@ -39,7 +41,7 @@ class Run:
     def generate(self, workers):
         """Gradients of the next len(workers) arrivals into the gradient buffers."""
         for j, i in enumerate(workers):
-            self.dev.grad_ptr(self.k + 1 + j, self.engine.saved_ptr(i), self.grads[j].data_ptr())
+            self.dev.grad_ptr(self.k + 1 + j, self._rows[i], self._grad_ptrs[j])
 
     def apply(self, workers):
         delays, launches = self.engine.push_batch(workers, self.grads[:len(workers)], return_launches=True)

@@ -944,6 +944,43 @@ def pin_learning_rate_schedule(make):
     assert np.allclose(th0.astype(np.float64) - o.get(THETA), e10 * g64 / (np.abs(g64) + 1e-8), rtol=1e-6)
 
 
+def pin_weight_decay_is_part_of_the_gradient(make):
+    """Appendix "Weight Decay": the decay element belongs to the gradient and is divided by the
+    Gap with it. A master with decay lambda fed g equals a master without decay fed
+    g + lambda * theta_k (theta_k = its parameters at that arrival), for every family; and the
+    textbook case: one worker, momentum SGD with weight_decay in torch."""
+    import torch
+    d, n, lam = 12, 3, 0.05
+    r = _rng(61)
+    th0 = _f32(r.normal(size=d))
+    sched = [0, 1, 2, 1, 0, 2, 0]
+    grads = [_f32(r.normal(size=d)) for _ in sched]
+    for variant in (ASGD, SA, GA, SA_GRAD, DANA_GA, ADAM_GA, GA_LAYER):
+        a = make(d, n, 0.1, 0.9, 0.999, variant, precision=64)
+        b = make(d, n, 0.1, 0.9, 0.999, variant, precision=64)
+        a.set_weight_decay(lam)
+        for o in (a, b):
+            o.set_params(th0)
+        for i, g in zip(sched, grads):
+            folded = g.astype(np.float64) + float(np.float32(lam)) * b.get(THETA)
+            # b is fed fp32 inputs: compare at fp32 resolution of the folded gradient
+            ta, tb = a.push(i, g), b.push(i, _f32(folded))
+            assert ta == tb
+            a.pull(i); b.pull(i)
+        assert np.allclose(a.get(THETA), b.get(THETA), rtol=2e-5, atol=2e-6), variant
+    p = torch.tensor(th0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([p], lr=float(np.float32(0.1)), momentum=float(np.float32(0.9)),
+                          weight_decay=float(np.float32(lam)))
+    o = make(d, 1, 0.1, 0.9, 0.999, GA, precision=64)
+    o.set_weight_decay(lam)
+    o.set_params(th0)
+    for g in grads:
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        o.push(0, g); o.pull(0)
+    assert np.allclose(o.get(THETA), p.detach().numpy(), rtol=1e-12, atol=1e-13)
+
+
 ALL_PINS = [
     pin_gap_is_one_where_copy_equals_master,
     pin_one_worker_is_heavy_ball,
@@ -971,4 +1008,5 @@ ALL_PINS = [
     pin_global_gap_definition,
     pin_layers_are_penalised_independently,
     pin_layer_gap_exact_brute_force,
+    pin_weight_decay_is_part_of_the_gradient,
 ]

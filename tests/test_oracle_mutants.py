@@ -49,15 +49,15 @@ MUTANTS = [
     ("m_weights_swapped", "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));",
      "m[j] = std::fma(one_minus_beta, m[j], beta * (v[j] * v[j]));"),
     ("m_from_raw_gradient", "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));",
-     "m[j] = std::fma(beta, m[j], one_minus_beta * ((T)grad[j] * (T)grad[j]));"),
+     "m[j] = std::fma(beta, m[j], one_minus_beta * (gw(grad, j) * gw(grad, j)));"),
     ("asgd_dampened", "v[j] = std::fma(gamma, v[j], g);\n                theta[j] = std::fma(-eta, v[j], theta[j]);",
      "v[j] = std::fma(gamma, v[j], ((T)1 - gamma) * g);\n                theta[j] = std::fma(-eta, v[j], theta[j]);"),
-    ("adam_order_uses_penalised_v", "const T u = std::fma(gamma, v[j], (T)grad[j]);",
+    ("adam_order_uses_penalised_v", "const T u = std::fma(gamma, v[j], gw(grad, j));",
      "const T u = v[j];"),
     ("set_params_keeps_momentum", "v[j] = 0;\n            m[j] = 0;", "m[j] = 0;"),
     # SA-Gradient and the DANA masters
-    ("sa_grad_multiplies", "const T g_tau = (T)grad[j] / (T)tau;", "const T g_tau = (T)grad[j] * (T)tau;"),
-    ("sa_grad_ignores_tau", "const T g_tau = (T)grad[j] / (T)tau;", "const T g_tau = (T)grad[j];"),
+    ("sa_grad_multiplies", "const T g_tau = gw(grad, j) / (T)tau;", "const T g_tau = gw(grad, j) * (T)tau;"),
+    ("sa_grad_ignores_tau", "const T g_tau = gw(grad, j) / (T)tau;", "const T g_tau = gw(grad, j);"),
     ("dana_estimate_sign", "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);",
      "saved[(size_t)i * d + j] = std::fma(eta_gamma, total, theta[j]);"),
     ("dana_estimate_without_gamma", "const T eta_gamma = eta * gamma;", "const T eta_gamma = eta;"),
@@ -91,8 +91,11 @@ MUTANTS = [
     ("adam_sa_multiplies", "first = one_minus_beta1 * (g / (T)tau);", "first = one_minus_beta1 * (g * (T)tau);"),
     ("adam_ga_divides_twice", "first = (one_minus_beta1 / G) * g;", "first = (one_minus_beta1 / G / G) * g;"),
     ("adam_ga_unpenalised", "first = (one_minus_beta1 / G) * g;", "first = one_minus_beta1 * g;"),
-    ("adam_ga_c_from_first_moment", "m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));\n            }\n            k_c += 1;\n        }\n        last_sum_gap",
-     "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));\n            }\n            k_c += 1;\n        }\n        last_sum_gap"),
+    ("adam_ga_c_from_first_moment", "m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));\n        }\n        if (variant == ADAM_GA && c_order == 0) k_c += 1;",
+     "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));\n        }\n        if (variant == ADAM_GA && c_order == 0) k_c += 1;"),
+    ("weight_decay_sign", "std::fma(wd, theta[j], (T)grad[j])", "std::fma(-wd, theta[j], (T)grad[j])"),
+    ("weight_decay_on_saved_copy_scale", "std::fma(wd, theta[j], (T)grad[j])", "std::fma(wd * wd, theta[j], (T)grad[j])"),
+    ("weight_decay_not_penalised", "const T g_hat = inv_gap * g;", "const T g_hat = inv_gap * (T)grad[j] + (g - (T)grad[j]);"),
     # layer-wise / global Gap
     ("layer_norm_is_l1", "dist2 += (double)diff * (double)diff;", "dist2 += std::fabs((double)diff);"),
     ("layer_norm_not_rooted", "const T dist = (T)std::sqrt(dist2);", "const T dist = (T)dist2;"),
@@ -104,7 +107,7 @@ MUTANTS = [
      "m_layer[p] = std::fma(beta, m_layer[p], one_minus_beta * (T)(norm2 / (double)(hi - lo)));"),
     ("layer_whole_vector_norm", "for (int64_t j = lo; j < hi; ++j) {\n                const T diff",
      "for (int64_t j = 0; j < d; ++j) {\n                const T diff"),
-    ("layer_unpenalised", "const T g_hat = inv_gap * (T)grad[j];\n                v[j]", "const T g_hat = (T)grad[j];\n                v[j]"),
+    ("layer_unpenalised", "const T g_hat = inv_gap * gw(grad, j);\n                v[j]", "const T g_hat = gw(grad, j);\n                v[j]"),
     ("dana_pull_forgets_iteration", "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);\n        }\n        iter[i] = k_done;",
      "saved[(size_t)i * d + j] = std::fma(-eta_gamma, total, theta[j]);\n        }"),
 ]
