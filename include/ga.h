@@ -89,7 +89,10 @@ enum {
     GA_OPT_WINDOW = 3,  /* 1..16 (default 16): most arrivals fused into one launch by
                            ga_push_batch. */
     GA_OPT_ADAM_BETA2 = 4, /* Adam variants: beta_2 in [0,1), default 0.999; before the first arrival */
-    GA_OPT_ADAM_EPS = 5    /* Adam variants: epsilon > 0, default 1e-8; before the first arrival */
+    GA_OPT_ADAM_EPS = 5,   /* Adam variants: epsilon > 0, default 1e-8; before the first arrival */
+    GA_OPT_WEIGHT_DECAY = 6 /* lambda >= 0 (default 0): the master adds lambda * theta_k to every arriving
+                              gradient before anything else, so the decay element is penalised with the
+                              gradient (Appendix "Weight Decay") */
 };
 
 #define GA_MAX_WINDOW 16

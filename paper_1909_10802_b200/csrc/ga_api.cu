@@ -53,6 +53,7 @@ struct ga_engine {
     int n_layers() const { return (int)layer_off.size() - 1; }
     float* sec = nullptr;         // Adam: second moment (vel holds the first moment, gamma is beta_1)
     float beta2 = 0.999f, adam_eps = 1e-8f;
+    float weight_decay = 0.f;
     std::vector<int64_t> iter;
     int64_t k_done = 0, k_c = 0;
     cudaStream_t stream = nullptr;
@@ -89,6 +90,7 @@ struct ga_engine {
         h.beta2 = beta2;
         h.one_minus_beta2 = (float)(1.0 - (double)beta2);
         h.adam_eps = adam_eps;
+        h.wd = weight_decay;
         return h;
     }
     // 1/(1-beta^k) for the C in force after k refreshes of m; 0 before the first (C = eta_max*eps)
@@ -163,14 +165,17 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
     const long long nvec = vec_end - vec_begin;
     long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
-    // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner
-    if (w.K == 1)
-        ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, 1, 0><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
-            e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
-    else   // Adam-GA is bound by its arithmetic, not by loads in flight: it keeps the register path
-        ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, GA_WINDOW_BATCH,
-                             (FAMILY == ga::ADAM && PENALTY == ga::PEN_GAP) ? 0 : GA_WINDOW_STAGES><<<(unsigned)blocks, ga::kThreads, 0, st>>>(
-            e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, vec_end, e->d, e->partials);
+    // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner.
+    // Adam-GA is bound by its arithmetic, not by loads in flight: it keeps the register path.
+    constexpr int ST = (FAMILY == ga::ADAM && PENALTY == ga::PEN_GAP) ? 0 : GA_WINDOW_STAGES;
+#define GA_LAUNCH(BATCH, STAGES_, WD_)                                                                          \
+    ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, BATCH, STAGES_, WD_>                            \
+        <<<(unsigned)blocks, ga::kThreads, 0, st>>>(e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, \
+                                                    vec_end, e->d, e->partials)
+    const bool wd = e->weight_decay != 0.f;
+    if (w.K == 1) { if (wd) GA_LAUNCH(1, 0, true); else GA_LAUNCH(1, 0, false); }
+    else { if (wd) GA_LAUNCH(GA_WINDOW_BATCH, ST, true); else GA_LAUNCH(GA_WINDOW_BATCH, ST, false); }
+#undef GA_LAUNCH
     if (STATS) {
         ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev);
     }
@@ -706,6 +711,10 @@ int ga_set_option(ga_engine* e, int key, double value) {
             if (e->k_done != 0) return fail(GA_ERR_STATE, "GA_OPT_ADAM_EPS can only change before the first arrival");
             e->adam_eps = (float)value;
             return GA_OK;
+        case GA_OPT_WEIGHT_DECAY:
+            if (!(value >= 0.0) || !std::isfinite(value)) return fail(GA_ERR_ARG, "GA_OPT_WEIGHT_DECAY must be >= 0");
+            e->weight_decay = (float)value;
+            return GA_OK;
         case GA_OPT_WINDOW:
             if (v < 1 || v > GA_MAX_WINDOW) return fail(GA_ERR_ARG, "GA_OPT_WINDOW must be in [1, %d]", GA_MAX_WINDOW);
             e->window = v;
@@ -745,7 +754,7 @@ struct StateHeader {
     int64_t d, n_workers, k_done, k_c;
     float lr, gamma, beta, eps;
     int32_t variant, c_order, fast_math, stats, window, reserved;
-    float beta2, adam_eps, lr_max, pad;
+    float beta2, adam_eps, lr_max, weight_decay;
 };
 
 size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
@@ -758,7 +767,7 @@ size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
     DeviceGuard guard(e->device);
     StateHeader h{};
     h.magic = kStateMagic; h.version = 2;
-    h.beta2 = e->beta2; h.adam_eps = e->adam_eps; h.lr_max = e->lr_max;
+    h.beta2 = e->beta2; h.adam_eps = e->adam_eps; h.lr_max = e->lr_max; h.weight_decay = e->weight_decay;
     h.d = e->d; h.n_workers = e->n_workers; h.k_done = e->k_done; h.k_c = e->k_c;
     h.lr = e->lr; h.gamma = e->gamma; h.beta = e->beta; h.eps = e->eps;
     h.variant = e->variant; h.c_order = e->c_order; h.fast_math = e->fast_math; h.stats = e->stats; h.window = e->window;
@@ -834,7 +843,7 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
     e->iter = iter;
     e->k_done = h.k_done; e->k_c = h.k_c;
     e->lr = h.lr; e->gamma = h.gamma; e->beta = h.beta; e->eps = h.eps;
-    e->beta2 = h.beta2; e->adam_eps = h.adam_eps; e->lr_max = h.lr_max;
+    e->beta2 = h.beta2; e->adam_eps = h.adam_eps; e->lr_max = h.lr_max; e->weight_decay = h.weight_decay;
     e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window;
     e->stats_valid = false;
     return GA_OK;

@@ -400,6 +400,27 @@ def test_sharded_runs_equal_the_whole(P):
     whole.close()
 
 
+@pytest.mark.parametrize("variant", ["GA", "SA", "DANA_GA", "ADAM_GA", "GA_LAYER"])
+def test_weight_decay(P, variant):
+    """GA_OPT_WEIGHT_DECAY: lambda * theta_k joins the gradient before the penalty."""
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("mini")
+    run = Run(wl, variant, 16, options={P.GA_OPT_WEIGHT_DECAY: 5e-4})
+    run.run()
+    o = oracle.Oracle(wl.d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, oracle.VARIANTS[variant])
+    if variant == "GA_LAYER":
+        o.set_layers(wl.seg_off)
+    o.set_weight_decay(5e-4)
+    o.set_params(wl.theta0())
+    for k, i in enumerate(wl.schedule(), start=1):
+        o.push(i, wl.grad(k, o.sent_f32(i)))
+        o.pull(i)
+    _compare_engine(P, run, o, label=f"{variant} with weight decay: ")
+    assert abs(P.unpack_state(run.engine.export_state())["weight_decay"] - np.float32(5e-4)) < 1e-10
+    assert run.engine._l.ga_set_option(run.engine._h, P.GA_OPT_WEIGHT_DECAY, -1.0) == P.GA_ERR_ARG
+    run.close()
+
+
 def test_c4_stragglers(P):
     import torch
     _sampled(P, "C4", "GA", 16).close()
