@@ -39,6 +39,7 @@ def _bind(path):
     lib.gao_set_eps.argtypes = [c.c_void_p, c.c_double]
     lib.gao_set_lr.argtypes = [c.c_void_p, c.c_double]
     lib.gao_set_weight_decay.argtypes = [c.c_void_p, c.c_double]
+    lib.gao_set_nesterov.argtypes = [c.c_void_p, c.c_int]
     lib.gao_set_params.argtypes = [c.c_void_p, c.c_void_p]
     lib.gao_pull.argtypes = [c.c_void_p, c.c_int]
     lib.gao_push.restype = c.c_int64
@@ -121,6 +122,9 @@ class Oracle:
         g, m = np.empty(n), np.empty(n)
         self._l.gao_layer_state(self._h, g.ctypes.data, m.ctypes.data)
         return g, m
+
+    def set_nesterov(self, on=True):
+        self._l.gao_set_nesterov(self._h, int(on))
 
     def set_weight_decay(self, wd):
         self._l.gao_set_weight_decay(self._h, wd)

@@ -102,6 +102,7 @@ struct Master {
     std::vector<double> last_layer_gap;
     std::vector<T> v2;          // Adam: second moment (the first moment lives in v; gamma is beta_1)
     T wd = 0;                   // weight decay lambda
+    int nesterov = 0;           // 1: Nesterov form of the momentum step
     T beta2 = (T)0.999f;        // Adam: beta_2
     T adam_eps = (T)1e-8f;      // Adam: epsilon
     std::vector<int64_t> iter;  // iteration array of the SA algorithm
@@ -114,6 +115,14 @@ struct Master {
     // the master forms it from its current parameters, g + lambda * theta_k (one FMA).
     T gw(const float* grad, int64_t j) const {
         return wd == (T)0 ? (T)grad[j] : std::fma(wd, theta[j], (T)grad[j]);
+    }
+
+    // The parameter step of the one-momentum-vector masters. Printed form: theta - eta v_{k+1}.
+    // Nesterov form (the paper's runs use "a NAG optimizer" but print no master-side formula;
+    // this is the form of the common framework optimisers): theta - eta (g_hat + gamma v_{k+1}).
+    T step(T th, T v_new, T g_pen, T e) const {
+        if (!nesterov) return std::fma(-e, v_new, th);
+        return std::fma(-e, std::fma(gamma, v_new, g_pen), th);
     }
 
     // 1 / (1 - beta^k) of the bias correction, k = refreshes of m so far (k >= 1).
@@ -167,7 +176,7 @@ struct Master {
             for (int64_t j = lo; j < hi; ++j) {
                 const T g_hat = inv_gap * gw(grad, j);
                 v[j] = std::fma(gamma, v[j], g_hat);
-                theta[j] = std::fma(-eta, v[j], theta[j]);
+                theta[j] = step(theta[j], v[j], g_hat, eta);
                 norm2 += (double)v[j] * (double)v[j];
             }
             m_layer[p] = std::fma(beta, m_layer[p], one_minus_beta * (T)norm2);
@@ -306,20 +315,20 @@ struct Master {
             for (int64_t j = 0; j < d; ++j) {
                 const T g_tau = gw(grad, j) / (T)tau;
                 v[j] = std::fma(gamma, v[j], g_tau);
-                theta[j] = std::fma(-eta, v[j], theta[j]);
+                theta[j] = step(theta[j], v[j], g_tau, eta);
             }
         } else if (variant == ASGD) {
             for (int64_t j = 0; j < d; ++j) {
                 const T g = gw(grad, j);
                 v[j] = std::fma(gamma, v[j], g);
-                theta[j] = std::fma(-eta, v[j], theta[j]);
+                theta[j] = step(theta[j], v[j], g, eta);
             }
         } else if (variant == SA) {
             const T eta_tau = eta / (T)tau;
             for (int64_t j = 0; j < d; ++j) {
                 const T g = gw(grad, j);
                 v[j] = std::fma(gamma, v[j], g);
-                theta[j] = std::fma(-eta_tau, v[j], theta[j]);
+                theta[j] = step(theta[j], v[j], g, eta_tau);
             }
         } else {
             const T one_minus_beta = (T)(1.0 - (double)beta);
@@ -341,7 +350,7 @@ struct Master {
                 const T inv_gap = (T)1 / G;       // the printed form: (1/G_k) (.) g
                 const T g_hat = inv_gap * g;
                 v[j] = std::fma(gamma, v[j], g_hat);
-                theta[j] = std::fma(-eta, v[j], theta[j]);
+                theta[j] = step(theta[j], v[j], g_hat, eta);
                 sum_gap += (double)G;
                 if ((double)G > max_gap) max_gap = (double)G;
             }
@@ -457,6 +466,11 @@ void gao_set_c_order(void* p, int c_order) {
 void gao_set_lr(void* p, double lr) {
     auto* h = (Handle*)p;
     if (h->precision == 32) h->f->eta = (float)lr; else h->g->eta = (double)(float)lr;
+}
+
+void gao_set_nesterov(void* p, int on) {
+    auto* h = (Handle*)p;
+    if (h->precision == 32) h->f->nesterov = on; else h->g->nesterov = on;
 }
 
 void gao_set_weight_decay(void* p, double wd) {

@@ -981,6 +981,41 @@ def pin_weight_decay_is_part_of_the_gradient(make):
     assert np.allclose(o.get(THETA), p.detach().numpy(), rtol=1e-12, atol=1e-13)
 
 
+def pin_nesterov_step(make):
+    """The Nesterov form of the momentum step, theta - eta (g_hat + gamma v_{k+1}): one worker
+    is torch.optim.SGD(nesterov=True); under GA the look-ahead uses the PENALISED gradient; the
+    momentum vector itself (and hence C) is that of the plain form."""
+    import torch
+    d, eta, gam = 15, 0.05, 0.9
+    r = _rng(71)
+    th0 = _f32(r.normal(size=d))
+    grads = [_f32(r.normal(size=d)) for _ in range(12)]
+    for variant in (ASGD, SA, GA, SA_GRAD, GA_LAYER):
+        p = torch.tensor(th0, dtype=torch.float64, requires_grad=True)
+        opt = torch.optim.SGD([p], lr=float(np.float32(eta)), momentum=float(np.float32(gam)), nesterov=True)
+        o = make(d, 1, eta, gam, 0.999, variant, precision=64)
+        o.set_nesterov()
+        o.set_params(th0)
+        for g in grads:
+            p.grad = torch.tensor(g, dtype=torch.float64)
+            opt.step()
+            o.push(0, g); o.pull(0)
+        assert np.allclose(o.get(THETA), p.detach().numpy(), rtol=1e-12, atol=1e-13), variant
+        assert np.allclose(o.get(V), opt.state[p]["momentum_buffer"].numpy(), rtol=1e-12, atol=1e-14)
+    # two workers under GA: theta moves by eta (g/G + gamma v_new), v_new = gamma v + g/G
+    a = make(d, 2, eta, gam, 0.999, GA, precision=64)
+    a.set_nesterov()
+    a.set_params(th0)
+    a.push(1, grads[0]); a.pull(1)
+    G, v_old, th_old = a.gap(0), a.get(V), a.get(THETA)
+    a.push(0, grads[1])
+    g_hat = grads[1].astype(np.float64) / G
+    v_new = float(np.float32(gam)) * v_old + g_hat
+    assert np.allclose(a.get(V), v_new, rtol=1e-13)
+    assert np.allclose(th_old - a.get(THETA), float(np.float32(eta)) * (g_hat + float(np.float32(gam)) * v_new), rtol=1e-11)
+    assert np.any(G > 1.5)
+
+
 ALL_PINS = [
     pin_gap_is_one_where_copy_equals_master,
     pin_one_worker_is_heavy_ball,
@@ -1009,4 +1044,5 @@ ALL_PINS = [
     pin_layers_are_penalised_independently,
     pin_layer_gap_exact_brute_force,
     pin_weight_decay_is_part_of_the_gradient,
+    pin_nesterov_step,
 ]

@@ -26,10 +26,15 @@ MUTANTS = [
     ("momentum_with_dampening", "v[j] = std::fma(gamma, v[j], g_hat);",
      "v[j] = std::fma(gamma, v[j], ((T)1 - gamma) * g_hat);"),
     ("momentum_dropped_in_ga", "v[j] = std::fma(gamma, v[j], g_hat);", "v[j] = g_hat;"),
-    ("step_sign", "theta[j] = std::fma(-eta, v[j], theta[j]);\n                sum_gap",
-     "theta[j] = std::fma(eta, v[j], theta[j]);\n                sum_gap"),
-    ("step_uses_gradient_not_v", "theta[j] = std::fma(-eta, v[j], theta[j]);\n                sum_gap",
-     "theta[j] = std::fma(-eta, g_hat, theta[j]);\n                sum_gap"),
+    ("step_sign", "theta[j] = step(theta[j], v[j], g_hat, eta);\n                sum_gap",
+     "theta[j] = step(theta[j], v[j], g_hat, -eta);\n                sum_gap"),
+    ("step_uses_gradient_not_v", "theta[j] = step(theta[j], v[j], g_hat, eta);\n                sum_gap",
+     "theta[j] = step(theta[j], g_hat, g_hat, eta);\n                sum_gap"),
+    ("plain_step_is_nesterov", "if (!nesterov) return std::fma(-e, v_new, th);", "if (nesterov) return std::fma(-e, v_new, th);"),
+    ("nesterov_without_gradient", "return std::fma(-e, std::fma(gamma, v_new, g_pen), th);",
+     "return std::fma(-e, gamma * v_new, th);"),
+    ("nesterov_lookahead_unscaled", "return std::fma(-e, std::fma(gamma, v_new, g_pen), th);",
+     "return std::fma(-e, v_new + g_pen, th);"),
     ("sa_multiplies_by_tau", "const T eta_tau = eta / (T)tau;", "const T eta_tau = eta * (T)tau;"),
     ("sa_ignores_tau", "const T eta_tau = eta / (T)tau;", "const T eta_tau = eta;"),
     ("sa_divides_gradient_twice", "const T eta_tau = eta / (T)tau;", "const T eta_tau = eta / (T)tau / (T)tau;"),
@@ -50,8 +55,8 @@ MUTANTS = [
      "m[j] = std::fma(one_minus_beta, m[j], beta * (v[j] * v[j]));"),
     ("m_from_raw_gradient", "m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));",
      "m[j] = std::fma(beta, m[j], one_minus_beta * (gw(grad, j) * gw(grad, j)));"),
-    ("asgd_dampened", "v[j] = std::fma(gamma, v[j], g);\n                theta[j] = std::fma(-eta, v[j], theta[j]);",
-     "v[j] = std::fma(gamma, v[j], ((T)1 - gamma) * g);\n                theta[j] = std::fma(-eta, v[j], theta[j]);"),
+    ("asgd_dampened", "v[j] = std::fma(gamma, v[j], g);\n                theta[j] = step(theta[j], v[j], g, eta);",
+     "v[j] = std::fma(gamma, v[j], ((T)1 - gamma) * g);\n                theta[j] = step(theta[j], v[j], g, eta);"),
     ("adam_order_uses_penalised_v", "const T u = std::fma(gamma, v[j], gw(grad, j));",
      "const T u = v[j];"),
     ("set_params_keeps_momentum", "v[j] = 0;\n            m[j] = 0;", "m[j] = 0;"),
