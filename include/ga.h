@@ -90,6 +90,11 @@ enum {
                            ga_push_batch. */
     GA_OPT_ADAM_BETA2 = 4, /* Adam variants: beta_2 in [0,1), default 0.999; before the first arrival */
     GA_OPT_ADAM_EPS = 5,   /* Adam variants: epsilon > 0, default 1e-8; before the first arrival */
+    GA_OPT_NESTEROV = 7,   /* 1: Nesterov form of the momentum step for GA_ASGD, GA_SA, GA_GA, GA_SA_GRAD and
+                              GA_GA_LAYER: theta <- theta - eta (g_hat + gamma v_{k+1}) with g_hat the penalised
+                              gradient. The paper's runs use "a NAG optimizer" (Section 6) but print no
+                              master-side formula; this is the form of the common framework optimisers.
+                              Default 0: the printed step theta - eta v_{k+1}. */
     GA_OPT_WEIGHT_DECAY = 6 /* lambda >= 0 (default 0): the master adds lambda * theta_k to every arriving
                               gradient before anything else, so the decay element is penalised with the
                               gradient (Appendix "Weight Decay") */

@@ -20,7 +20,7 @@ LIB_PATH = os.environ.get("GA_LIBRARY") or os.path.join(_HERE, "libga.so")   # G
 GA_OK, GA_ERR_ARG, GA_ERR_STATE, GA_ERR_OOM, GA_ERR_CUDA = 0, -1, -2, -3, -4
 GA_THETA, GA_V, GA_M, GA_C, GA_V2 = 0, 1, 2, 3, 4
 (GA_OPT_C_ORDER, GA_OPT_MATH, GA_OPT_STATS, GA_OPT_WINDOW, GA_OPT_ADAM_BETA2, GA_OPT_ADAM_EPS,
- GA_OPT_WEIGHT_DECAY) = range(7)
+ GA_OPT_WEIGHT_DECAY, GA_OPT_NESTEROV) = range(8)
 GA_MAX_WINDOW = 16
 GA_NOALLOC_MAX_PARAMS = 1 << 28
 VARIANTS = {"ASGD": GA_ASGD, "SA": GA_SA, "GA": GA_GA, "SA_GRAD": GA_SA_GRAD, "DANA": GA_DANA,
@@ -290,7 +290,7 @@ def unpack_state(blob):
     import numpy as np
     hs = struct.calcsize(_HEADER)
     (magic, version, d, n, k_done, k_c, lr, gamma, beta, eps, variant, c_order, fast_math, stats,
-     window, _, beta2, adam_eps, lr_max, weight_decay) = struct.unpack_from(_HEADER, blob, 0)
+     window, nesterov, beta2, adam_eps, lr_max, weight_decay) = struct.unpack_from(_HEADER, blob, 0)
     if magic != _MAGIC or version != 2:
         raise ValueError("not a Gap-Aware master checkpoint")
     off = hs
@@ -301,7 +301,7 @@ def unpack_state(blob):
     rows = 3 + n * (2 if dana else 1) + (1 if adam else 0)
     vecs = np.frombuffer(blob, dtype=np.float32, count=rows * d, offset=off).reshape(rows, d).copy()
     extra = {"v_workers": vecs[3 + n:]} if dana else {"v2": vecs[3 + n]} if adam else {}
-    extra.update(beta2=beta2, adam_eps=adam_eps, lr_max=lr_max, weight_decay=weight_decay)
+    extra.update(beta2=beta2, adam_eps=adam_eps, lr_max=lr_max, weight_decay=weight_decay, nesterov=nesterov)
     if variant == GA_GA_LAYER:
         at = off + 4 * rows * d
         nl = int(np.frombuffer(blob, dtype=np.int64, count=1, offset=at)[0])
@@ -319,7 +319,7 @@ def pack_state(st):
     import numpy as np
     head = struct.pack(_HEADER, _MAGIC, 2, st["d"], st["n_workers"], st["k_done"], st["k_c"], st["lr"],
                        st["momentum"], st["c_beta"], st["eps"], st["variant"], st["c_order"],
-                       st["fast_math"], st["stats"], st["window"], 0, st.get("beta2", 0.999),
+                       st["fast_math"], st["stats"], st["window"], st.get("nesterov", 0), st.get("beta2", 0.999),
                        st.get("adam_eps", 1e-8), st.get("lr_max", st["lr"]), st.get("weight_decay", 0.0))
     parts = [head, np.ascontiguousarray(st["iter"], dtype=np.int64).tobytes()]
     for name in ("theta", "v", "m", "saved") + tuple(x for x in ("v_workers", "v2") if x in st):

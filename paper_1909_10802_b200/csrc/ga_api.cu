@@ -54,6 +54,7 @@ struct ga_engine {
     float* sec = nullptr;         // Adam: second moment (vel holds the first moment, gamma is beta_1)
     float beta2 = 0.999f, adam_eps = 1e-8f;
     float weight_decay = 0.f;
+    int nesterov = 0;
     std::vector<int64_t> iter;
     int64_t k_done = 0, k_c = 0;
     cudaStream_t stream = nullptr;
@@ -91,6 +92,7 @@ struct ga_engine {
         h.one_minus_beta2 = (float)(1.0 - (double)beta2);
         h.adam_eps = adam_eps;
         h.wd = weight_decay;
+        h.nesterov = nesterov;
         return h;
     }
     // 1/(1-beta^k) for the C in force after k refreshes of m; 0 before the first (C = eta_max*eps)
@@ -172,7 +174,7 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
     ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, BATCH, STAGES_, WD_>                            \
         <<<(unsigned)blocks, ga::kThreads, 0, st>>>(e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, \
                                                     vec_end, e->d, e->partials)
-    const bool wd = e->weight_decay != 0.f;
+    const bool wd = e->weight_decay != 0.f || e->nesterov;   // the instantiations with the extras
     if (w.K == 1) { if (wd) GA_LAUNCH(1, 0, true); else GA_LAUNCH(1, 0, false); }
     else { if (wd) GA_LAUNCH(GA_WINDOW_BATCH, ST, true); else GA_LAUNCH(GA_WINDOW_BATCH, ST, false); }
 #undef GA_LAUNCH
@@ -711,6 +713,12 @@ int ga_set_option(ga_engine* e, int key, double value) {
             if (e->k_done != 0) return fail(GA_ERR_STATE, "GA_OPT_ADAM_EPS can only change before the first arrival");
             e->adam_eps = (float)value;
             return GA_OK;
+        case GA_OPT_NESTEROV:
+            if (v != 0 && v != 1) return fail(GA_ERR_ARG, "GA_OPT_NESTEROV must be 0 or 1");
+            if (v && (e->is_dana() || e->is_adam()))
+                return fail(GA_ERR_STATE, "the Nesterov step exists for the one-momentum-vector variants only");
+            e->nesterov = v;
+            return GA_OK;
         case GA_OPT_WEIGHT_DECAY:
             if (!(value >= 0.0) || !std::isfinite(value)) return fail(GA_ERR_ARG, "GA_OPT_WEIGHT_DECAY must be >= 0");
             e->weight_decay = (float)value;
@@ -753,7 +761,7 @@ struct StateHeader {
     uint32_t magic, version;
     int64_t d, n_workers, k_done, k_c;
     float lr, gamma, beta, eps;
-    int32_t variant, c_order, fast_math, stats, window, reserved;
+    int32_t variant, c_order, fast_math, stats, window, nesterov;
     float beta2, adam_eps, lr_max, weight_decay;
 };
 
@@ -770,7 +778,7 @@ size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
     h.beta2 = e->beta2; h.adam_eps = e->adam_eps; h.lr_max = e->lr_max; h.weight_decay = e->weight_decay;
     h.d = e->d; h.n_workers = e->n_workers; h.k_done = e->k_done; h.k_c = e->k_c;
     h.lr = e->lr; h.gamma = e->gamma; h.beta = e->beta; h.eps = e->eps;
-    h.variant = e->variant; h.c_order = e->c_order; h.fast_math = e->fast_math; h.stats = e->stats; h.window = e->window;
+    h.variant = e->variant; h.c_order = e->c_order; h.fast_math = e->fast_math; h.stats = e->stats; h.window = e->window; h.nesterov = e->nesterov;
     char* p = (char*)buf_host;
     std::memcpy(p, &h, sizeof h); p += sizeof h;
     std::memcpy(p, e->iter.data(), sizeof(int64_t) * e->n_workers); p += sizeof(int64_t) * e->n_workers;
@@ -844,7 +852,7 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
     e->k_done = h.k_done; e->k_c = h.k_c;
     e->lr = h.lr; e->gamma = h.gamma; e->beta = h.beta; e->eps = h.eps;
     e->beta2 = h.beta2; e->adam_eps = h.adam_eps; e->lr_max = h.lr_max; e->weight_decay = h.weight_decay;
-    e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window;
+    e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window; e->nesterov = h.nesterov;
     e->stats_valid = false;
     return GA_OK;
 }

@@ -108,7 +108,8 @@ ga_layer_update_kernel(float* __restrict__ theta, float* __restrict__ vel, const
     auto one = [&](float& th, float& v, float g) {
         if (h.wd != 0.0f) g = __fmaf_rn(h.wd, th, g);      // decay element: part of the gradient
         v = __fmaf_rn(h.gamma, v, __fmul_rn(inv, g));      // (1/G_p) g, then the momentum step
-        th = __fmaf_rn(-eta, v, th);
+        if (h.nesterov) th = __fmaf_rn(-eta, __fmaf_rn(h.gamma, v, __fmul_rn(inv, g)), th);
+        else th = __fmaf_rn(-eta, v, th);
         acc += (double)v * (double)v;
     };
     auto scalar = [&](long long i) {

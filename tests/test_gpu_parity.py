@@ -421,6 +421,30 @@ def test_weight_decay(P, variant):
     run.close()
 
 
+@pytest.mark.parametrize("variant", ["GA", "SA", "ASGD", "SA_GRAD", "GA_LAYER"])
+def test_nesterov_step(P, variant):
+    """GA_OPT_NESTEROV (with weight decay on top, the usual recipe of the paper's CIFAR runs)."""
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("mini")
+    run = Run(wl, variant, 16, options={P.GA_OPT_NESTEROV: 1, P.GA_OPT_WEIGHT_DECAY: 1e-4})
+    run.run()
+    o = oracle.Oracle(wl.d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, oracle.VARIANTS[variant])
+    if variant == "GA_LAYER":
+        o.set_layers(wl.seg_off)
+    o.set_nesterov()
+    o.set_weight_decay(1e-4)
+    o.set_params(wl.theta0())
+    for k, i in enumerate(wl.schedule(), start=1):
+        o.push(i, wl.grad(k, o.sent_f32(i)))
+        o.pull(i)
+    _compare_engine(P, run, o, label=f"{variant}, Nesterov: ")
+    assert P.unpack_state(run.engine.export_state())["nesterov"] == 1
+    run.close()
+    dana = P.Engine(64, 2, 0.1, 0.9, 0.999, P.GA_DANA)
+    assert dana._l.ga_set_option(dana._h, P.GA_OPT_NESTEROV, 1.0) == P.GA_ERR_STATE
+    dana.close()
+
+
 def test_c4_stragglers(P):
     import torch
     _sampled(P, "C4", "GA", 16).close()
