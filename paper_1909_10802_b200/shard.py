@@ -34,3 +34,16 @@ def assert_same_schedule(schedule, dist):
     dist.all_gather_object(all_, mine)
     if any(x != mine for x in all_):
         raise RuntimeError("ranks disagree on the arrival schedule")
+
+
+def combine_gap_stats(sum_gap, max_gap, dist):
+    """Gap statistics of a sharded master: every rank holds the sum and maximum of the Gap over
+    its own range (ga_get_stats); the whole vector's are the sum of sums and the max of maxima.
+    These two scalars per arrival are the only values ranks ever exchange, and only for logging."""
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    s = torch.tensor([sum_gap], dtype=torch.float64, device=dev)
+    m = torch.tensor([max_gap], dtype=torch.float64, device=dev)
+    dist.all_reduce(s, op=dist.ReduceOp.SUM)
+    dist.all_reduce(m, op=dist.ReduceOp.MAX)
+    return float(s.item()), float(m.item())

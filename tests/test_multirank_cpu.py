@@ -18,7 +18,7 @@ def _free_port():
 def _rank(rank, world, port, out_dir):
     import torch
     import torch.distributed as dist
-    from paper_1909_10802_b200.shard import assert_same_schedule, shard_range
+    from paper_1909_10802_b200.shard import assert_same_schedule, combine_gap_stats, shard_range
     from tests.oracle_run import run_oracle
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     dist.init_process_group("gloo", rank=rank, world_size=world)
@@ -31,6 +31,8 @@ def _rank(rank, world, port, out_dir):
     all_delays = [None] * world
     dist.all_gather_object(all_delays, delays)
     assert all(x == delays for x in all_delays)
+    total, biggest = combine_gap_stats(*o.stats(), dist)      # statistics of the last arrival
+    np.save(os.path.join(out_dir, f"stats_{rank}.npy"), np.array([total, biggest]))
     np.save(os.path.join(out_dir, f"theta_{rank}.npy"), o.get(o.THETA))
     np.save(os.path.join(out_dir, f"m_{rank}.npy"), o.get(o.M))
     # a rank with a different schedule is detected
@@ -56,3 +58,7 @@ def test_two_ranks_equal_one(tmp_path):
     theta = np.concatenate([np.load(tmp_path / f"theta_{r}.npy") for r in range(world)])
     m = np.concatenate([np.load(tmp_path / f"m_{r}.npy") for r in range(world)])
     assert np.array_equal(theta, full.get(full.THETA)) and np.array_equal(m, full.get(full.M))
+    want_sum, want_max = full.stats()
+    for r in range(world):
+        got_sum, got_max = np.load(tmp_path / f"stats_{r}.npy")
+        assert abs(got_sum - want_sum) <= 1e-12 * want_sum and got_max == want_max
