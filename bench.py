@@ -288,7 +288,7 @@ def run_ours(args):
 
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, run, wl, world, dist if world > 1 else None, barrier)
+        e2e = run_e2e(args, run, wl, base, world, dist if world > 1 else None, barrier)
     run.close()
     torch.cuda.empty_cache()
 
@@ -319,12 +319,12 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def run_e2e(args, run, wl, world, dist, barrier):
+def run_e2e(args, run, wl, base, world, dist, barrier):
     """Same metric through ga_push_batch_host: gradients start in pinned host memory and the
     parameters sent back to each worker end in pinned host memory, copies inside the timed region."""
     import torch
     k = min(args.e2e_window, args.window)
-    wins = bench_windows(wl, k, args.e2e_steps + 1)
+    wins = bench_windows(base, k, args.e2e_steps + 1)      # the replicated schedule
     grads = [torch.empty(wl.d, dtype=torch.float32).pin_memory() for _ in range(k)]
     outs = [torch.empty(wl.d, dtype=torch.float32).pin_memory() for _ in range(k)]
     for j, g in enumerate(grads):                     # synthetic gradients, generated on the device
