@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--math", default="exact", choices=["exact", "fast"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--e2e-window", type=int, default=8)
+    ap.add_argument("--probe-hbm", action="store_true",
+                    help="print the bandwidth of plain torch kernels (copy, add, sum, fill) on this GPU and exit")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-params", type=int, default=4_000_000)
@@ -355,8 +357,36 @@ def run_e2e(args, run, wl, base, world, dist, barrier):
             "note": "ga_push_batch_host: pinned host gradients in, sent parameters out, chunked overlap"}
 
 
+def probe_hbm():
+    """Context for the roofline denominator: what library kernels with simple read/write mixes
+    reach on this GPU (4 GiB fp32 vectors, best of 10, CUDA events)."""
+    import torch
+    n = 1 << 30
+    a, b = torch.randn(n, device="cuda"), torch.randn(n, device="cuda")
+    c = torch.empty_like(a)
+    out = {}
+    for name, fn, nbytes in (("copy_1r1w", lambda: c.copy_(a), 8 * n), ("add_2r1w", lambda: torch.add(a, b, out=c), 12 * n),
+                             ("sum_read_only", lambda: a.sum(), 4 * n), ("fill_write_only", lambda: c.fill_(1.0), 4 * n)):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        out[name] = round(nbytes / best / 1e6, 1)
+    print(json.dumps({"probe": "hbm_gbs_of_torch_kernels", **out}), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.probe_hbm:
+        probe_hbm()
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
