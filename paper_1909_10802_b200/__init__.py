@@ -219,6 +219,15 @@ class Engine:
         launches = _check(self._l.ga_push_batch(self._h, sched, ptrs, k, delays))
         return (list(delays), launches) if return_launches else list(delays)
 
+    def push_batch_raw(self, sched_array, ptr_array, k, delays_array):
+        """ga_push_batch on caller-kept ctypes arrays (c_int[k], c_void_p[k], c_int64[k]): the
+        lean path for loops over small vectors, where building arrays per call would dominate.
+        Returns the number of launches."""
+        rc = self._l.ga_push_batch(self._h, sched_array, ptr_array, k, delays_array)
+        if rc < 0:
+            raise GaError(rc, last_error())
+        return rc
+
     def push_batch_host(self, schedule, grads_host, sent_out_host=None):
         """grads_host / sent_out_host: CPU tensors (pinned for speed) of n_params floats."""
         k = len(schedule)

@@ -4,6 +4,8 @@ For every window of the arrival schedule the stand-in gradients are generated on
 from the parameters each worker was last sent, then the window goes to ga_push_batch. The
 generators come from the `workloads` module; no update arithmetic happens here.
 """
+import ctypes
+
 import workloads as W
 
 from . import Engine, GA_MAX_WINDOW, GA_OPT_WINDOW, VARIANTS
@@ -34,6 +36,10 @@ class Run:
         self.grads = [torch.empty(self.n, dtype=torch.float32, device=torch_device) for _ in range(window)]
         self._rows = [self.engine.saved_ptr(i) for i in range(wl.n_workers)]   # stable for the engine's life
         self._grad_ptrs = [g.data_ptr() for g in self.grads]
+        # arrays handed to ga_push_batch, kept across calls (the gradient buffers never move)
+        self._sched = (ctypes.c_int * window)()
+        self._ptrs = (ctypes.c_void_p * window)(*self._grad_ptrs)
+        self._delays = (ctypes.c_int64 * window)()
         self.k = 0            # arrivals applied
         self.delays = []
         self.launches = 0
@@ -44,10 +50,12 @@ class Run:
             self.dev.grad_ptr(self.k + 1 + j, self._rows[i], self._grad_ptrs[j])
 
     def apply(self, workers):
-        delays, launches = self.engine.push_batch(workers, self.grads[:len(workers)], return_launches=True)
-        self.k += len(workers)
+        n = len(workers)
+        self._sched[:n] = workers
+        self.launches += self.engine.push_batch_raw(self._sched, self._ptrs, n, self._delays)
+        delays = self._delays[:n]
+        self.k += n
         self.delays += delays
-        self.launches += launches
         return delays
 
     def step(self, workers):

@@ -396,6 +396,9 @@ class DeviceWorkload:
         self.seg_off = torch.from_numpy(wl.seg_off).to(torch_device)
         self.seg_sigma = torch.from_numpy(wl.seg_sigma).to(torch_device)
         self.lib = cuda_lib()
+        self._spec_ref = ctypes.byref(wl.spec)
+        self._seg_off_p = ctypes.c_void_p(self.seg_off.data_ptr())
+        self._seg_sigma_p = ctypes.c_void_p(self.seg_sigma.data_ptr())
 
     def _stream(self):
         return ctypes.c_void_p(self._torch.cuda.current_stream().cuda_stream)
@@ -408,9 +411,8 @@ class DeviceWorkload:
         return out
 
     def grad_ptr(self, k, sent_ptr, out_ptr):
-        rc = self.lib.wl_cuda_grad(ctypes.byref(self.wl.spec), ctypes.c_void_p(self.seg_off.data_ptr()),
-                                   ctypes.c_void_p(self.seg_sigma.data_ptr()), k, self.j0, self.n,
-                                   ctypes.c_void_p(sent_ptr), ctypes.c_void_p(out_ptr), self._stream())
+        rc = self.lib.wl_cuda_grad(self._spec_ref, self._seg_off_p, self._seg_sigma_p, k, self.j0, self.n,
+                                   sent_ptr, out_ptr, self._stream())
         if rc:
             raise RuntimeError(f"wl_cuda_grad: CUDA error {rc}")
 
