@@ -458,6 +458,15 @@ def test_c5_transformer_lm_full_size(P):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("variant", ["DANA_GA", "ADAM_GA", "SA_GRAD"])
+def test_c5_full_size_other_masters(P, variant):
+    """150M parameters, 32 workers, K = 16 for the appendix's masters (DANA-GA adds 19 GB of
+    per-worker momentum); 96 arrivals, sampled parameters against the oracle."""
+    import torch
+    _sampled(P, "C5", variant, 16, n_arrivals=96).close()
+    torch.cuda.empty_cache()
+
+
 # ----------------------------------------------------------------------------- single calls
 def _small_engine(P, d=5003, n=4, variant=None, seed=5):
     import torch
