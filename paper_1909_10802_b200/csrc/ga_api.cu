@@ -375,7 +375,7 @@ const char* ga_last_error(void) { return g_error.c_str(); }
 
 ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, float c_beta, int variant) {
     g_error.clear();
-    if (n_params == 0 || n_params > (size_t)1 << 40) { fail(GA_ERR_ARG, "n_params out of range"); return nullptr; }
+    if (n_params == 0 || n_params > (size_t)1 << 34) { fail(GA_ERR_ARG, "n_params out of range"); return nullptr; }
     if (n_workers <= 0 || n_workers > 65536) { fail(GA_ERR_ARG, "n_workers out of range"); return nullptr; }
     if (!(lr > 0.f) || !std::isfinite(lr)) { fail(GA_ERR_ARG, "lr must be positive and finite"); return nullptr; }
     if (!(std::fabs(momentum) < 1.f)) { fail(GA_ERR_ARG, "|momentum| must be < 1"); return nullptr; }
