@@ -631,6 +631,68 @@ def test_single_arrival_against_fp64(P, math_mode):
         eng.close()
 
 
+@pytest.mark.parametrize("variant", ["GA", "DANA_GA", "ADAM_GA", "SA_GRAD", "GA_LAYER"])
+def test_extreme_values_round_like_the_oracle(P, variant):
+    """States and gradients spanning the whole fp32 range -- subnormals, zeros of both signs,
+    1e-42 .. 1e38, infinities, NaNs -- imported into both sides; a window of three arrivals must
+    still agree element for element (the IEEE division / square-root / reciprocal paths and
+    their zero shortcuts are all exercised)."""
+    import torch
+    d, n = 60_000, 3
+    rng = np.random.default_rng(99)
+
+    def wild(nonneg=False):
+        x = (10.0 ** rng.uniform(-44, 38, size=d)) * (1 if nonneg else rng.choice([-1.0, 1.0], size=d))
+        x = x.astype(np.float32)
+        kind = rng.integers(0, 40, size=d)
+        x[kind == 0] = 0.0
+        x[kind == 1] = 0.0 if nonneg else -0.0
+        x[kind == 2] = np.inf
+        x[kind == 3] = np.inf if nonneg else -np.inf
+        x[kind == 4] = np.nan
+        x[kind == 5] = np.float32(1e-45)          # smallest subnormal
+        return x
+
+    var = oracle.VARIANTS[variant]
+    o = oracle.Oracle(d, n, 0.1, 0.9, 0.999, var)
+    eng = P.Engine(d, n, 0.1, 0.9, 0.999, var)
+    theta, v, m = wild(), wild(), wild(nonneg=True)
+    saved = np.stack([wild() for _ in range(n)])
+    saved[0, ::3] = theta[::3]                     # plenty of exact "copy equals master"
+    iters = np.array([2, 0, 4], dtype=np.int64)
+    extra = {}
+    if variant == "DANA_GA":
+        extra = dict(v_workers=np.stack([wild() for _ in range(n)]))
+    if variant == "ADAM_GA":
+        extra = dict(v_workers=wild(nonneg=True))
+    o.set_state(theta, v, m, saved, iters, 5, 5, **extra)
+    if variant == "GA_LAYER":                      # three layers; their m_p start at 0 on both sides
+        o.set_layers([0, 7, 30_001, d])
+        eng.set_layers([0, 7, 30_001, d])
+    st = P.unpack_state(eng.export_state())
+    st.update(theta=theta, v=v, m=m, saved=saved, iter=iters, k_done=5, k_c=5)
+    if variant == "DANA_GA":
+        st["v_workers"] = extra["v_workers"]
+    if variant == "ADAM_GA":
+        st["v2"] = extra["v_workers"]
+    eng.import_state(P.pack_state(st))
+    grads = [wild() for _ in range(3)]
+    sched = [1, 0, 2]
+    assert eng.push_batch(sched, [torch.from_numpy(g).cuda() for g in grads]) == o.push_batch(sched, grads)
+    pairs = [(P.GA_THETA, o.get(o.THETA)), (P.GA_V, o.get(o.V))]
+    if variant in ("GA", "DANA_GA", "ADAM_GA"):
+        pairs.append((P.GA_M, o.get(o.M)))
+    if variant == "ADAM_GA":
+        pairs.append((P.GA_V2, o.second_moment()))
+    for which, ref in pairs:
+        got = _np(eng.get(which))
+        bad = ~((got == ref.astype(np.float32)) | (np.isnan(got) & np.isnan(ref)))
+        assert not bad.any(), (variant, which, int(bad.sum()), got[bad][:4], ref[bad][:4])
+    for i in range(n):
+        assert _same(_np(eng.saved(i)), o.saved(i))
+    eng.close()
+
+
 # ----------------------------------------------------------------------------- errors
 def test_bad_arguments_return_errors(P):
     import ctypes
