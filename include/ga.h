@@ -81,7 +81,8 @@ enum {
     GA_OPT_MATH = 1,    /* 0 (default): every operation IEEE round-to-nearest, in the order of
                            the algorithms. 1: fast: approximate reciprocal and square root, one
                            division per element (g*C/(|theta-theta^i|+C)); a few ulp off. Applies
-                           to GA_GA and GA_DANA_GA; every other variant is always exact. */
+                           to GA_GA, GA_DANA_GA and GA_ADAM_GA (there also to Adam's own root and
+                           division); every other variant is always exact. */
     GA_OPT_STATS = 2,   /* 1: every GA push also reduces sum and max of the Gap over all
                            parameters (the quantity the paper logs per epoch, Appendix
                            "Gap and Delay"); read with ga_get_stats. Default 0. Not computed by

@@ -168,8 +168,8 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
     long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
     // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner.
-    // Adam-GA is bound by its arithmetic, not by loads in flight: it keeps the register path.
-    constexpr int ST = (FAMILY == ga::ADAM && PENALTY == ga::PEN_GAP) ? 0 : GA_WINDOW_STAGES;
+    // Exact Adam-GA is bound by its arithmetic, not by loads in flight: it keeps the register path.
+    constexpr int ST = (FAMILY == ga::ADAM && PENALTY == ga::PEN_GAP && EXACT) ? 0 : GA_WINDOW_STAGES;
 #define GA_LAUNCH(BATCH, STAGES_, WD_)                                                                          \
     ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, BATCH, STAGES_, WD_>                            \
         <<<(unsigned)blocks, ga::kThreads, 0, st>>>(e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, \
@@ -186,7 +186,7 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
 template <int FAMILY>
 void launch_family(ga_engine* e, const ga::Window& w, long long vb, long long ve, cudaStream_t st, bool stats) {
     if (e->is_gap()) {
-        const bool exact = !e->fast_math || FAMILY == ga::ADAM;   // Adam has no fast-math form
+        const bool exact = !e->fast_math;
 #define GA_CASE(EX, CO, ST) launch_window_t<FAMILY, ga::PEN_GAP, EX, CO, ST>(e, w, vb, ve, st)
         if (exact) {
             if (e->c_order == 0) { if (stats) GA_CASE(true, 0, true); else GA_CASE(true, 0, false); }

@@ -603,6 +603,33 @@ def test_host_buffer_path_equals_device_path(P):
 
 
 # ----------------------------------------------------------------------------- fp64 and fast mode
+def test_adam_ga_fast_math_single_arrival(P):
+    """Adam-GA's fast form against the fp64 oracle, one arrival from an identical fp32 state."""
+    import torch
+    wl = W.Workload(name="adamfast", segments=[30_000], n_workers=4, arrivals=40, schedule_kind="ticks",
+                    seed=321, lr=0.01)
+    sched = wl.schedule()
+    for start in (0, 25):
+        o32, _, _ = run_oracle(wl, "ADAM_GA", n_arrivals=start)
+        state = o32.state()
+        o64 = oracle.Oracle(wl.d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, oracle.ADAM_GA, precision=64)
+        o64.set_state(*state[:7], v_workers=state[7])
+        eng = P.Engine(wl.d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, P.GA_ADAM_GA)
+        eng.set_option(P.GA_OPT_MATH, 1)
+        st = P.unpack_state(eng.export_state())
+        st.update(theta=state[0], v=state[1], m=state[2], saved=state[3], iter=state[4], k_done=state[5],
+                  k_c=state[6], v2=state[7])
+        eng.import_state(P.pack_state(st))
+        i = sched[start]
+        g = wl.grad(start + 1, o32.sent_f32(i))
+        assert eng.push_batch([i], [torch.from_numpy(g).cuda()]) == [o64.push(i, g)]
+        for which, ref in ((P.GA_THETA, o64.get(o64.THETA)), (P.GA_V, o64.get(o64.V)), (P.GA_V2, o64.second_moment()),
+                           (P.GA_M, o64.get(o64.M))):
+            got = _np(eng.get(which))
+            assert within(got, ref, TOL), (start, which, worst(got, ref))
+        eng.close()
+
+
 @pytest.mark.parametrize("math_mode", [0, 1])
 def test_single_arrival_against_fp64(P, math_mode):
     """From one fp32 state, one arrival on the GPU (exact or fast math) and in the fp64 oracle."""
