@@ -16,7 +16,12 @@ def build(force=False, verbose=False):
         return LIB
     tmp = f"{LIB}.{os.getpid()}.tmp"
     cmd = ["nvcc", *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp, *SOURCES]
-    subprocess.check_call(cmd)
+    try:
+        subprocess.check_call(cmd)
+    except (OSError, subprocess.CalledProcessError):
+        if os.path.exists(LIB) and not force:   # no nvcc here: keep the library that travelled with the tree
+            return LIB
+        raise
     os.replace(tmp, LIB)
     return LIB
 
