@@ -83,18 +83,20 @@ enum {
                            division per element (g*C/(|theta-theta^i|+C)); a few ulp off. Applies
                            to GA_GA, GA_DANA_GA and GA_ADAM_GA (there also to Adam's own root and
                            division); every other variant is always exact. */
-    GA_OPT_STATS = 2,   /* 1: every GA push also reduces sum and max of the Gap over all
-                           parameters (the quantity the paper logs per epoch, Appendix
-                           "Gap and Delay"); read with ga_get_stats. Default 0. Not computed by
-                           ga_push_batch_host, nor for GA_GA_LAYER (see ga_get_layer_state). */
+    GA_OPT_STATS = 2,   /* 1: every arrival of GA_GA, GA_DANA_GA and GA_ADAM_GA also reduces the sum
+                           and the maximum of the Gap over all parameters (the average Gap is what
+                           Appendix "Gap and Delay" logs); read with ga_get_stats_window or
+                           ga_get_stats. Default 0. Not computed for GA_GA_LAYER, which has one Gap
+                           per layer (see ga_get_layer_state). */
     GA_OPT_WINDOW = 3,  /* 1..16 (default 16): most arrivals fused into one launch by
                            ga_push_batch. */
     GA_OPT_ADAM_BETA2 = 4, /* Adam variants: beta_2 in [0,1), default 0.999; before the first arrival */
     GA_OPT_ADAM_EPS = 5,   /* Adam variants: epsilon > 0, default 1e-8; before the first arrival */
     GA_OPT_NESTEROV = 7,   /* 1: Nesterov form of the momentum step for GA_ASGD, GA_SA, GA_GA, GA_SA_GRAD and
                               GA_GA_LAYER: theta <- theta - eta (g_hat + gamma v_{k+1}) with g_hat the penalised
-                              gradient. The paper's runs use "a NAG optimizer" (Section 6) but print no
-                              master-side formula; this is the form of the common framework optimisers.
+                              gradient. Section 6 says the experiments ran Nesterov momentum, but no
+                              master algorithm is printed in that form; this is the form of the common
+                              framework optimisers.
                               Default 0: the printed step theta - eta v_{k+1}. */
     GA_OPT_WEIGHT_DECAY = 6 /* lambda >= 0 (default 0): the master adds lambda * theta_k to every arriving
                               gradient before anything else, so the decay element is penalised with the
@@ -107,7 +109,9 @@ enum {
  * C algorithm), momentum is gamma (|gamma| < 1; Section 3, no dampening), c_beta is beta_1 of
  * Algorithm "C Coefficient Calculation" (0 <= c_beta < 1; the paper uses 0.999; eps is 1e-8).
  * All state starts at 0: theta = v = m = 0, every saved copy = 0, no arrivals, iter[] = 0.
- * Returns NULL on invalid arguments or allocation failure (see ga_last_error). */
+ * lr must be large enough that lr * 1e-8, the smallest value C can take, does not round to zero
+ * in fp32 (lr above about 1.5e-37). Returns NULL on invalid arguments or allocation failure (see
+ * ga_last_error). */
 ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, float c_beta,
                      int variant);
 
@@ -118,8 +122,9 @@ void ga_destroy(ga_engine* e);
 int ga_set_stream(ga_engine* e, void* cuda_stream);
 
 /* Learning rate eta_k for the arrivals that follow (decay, warm-up: Appendix "Hyperparameters").
- * eta_max of the C algorithm stays the rate given to ga_create ("usually eta_max = eta_1"), so
- * the Gap penalty relaxes as the rate decays (Section 5.1). lr must be positive and finite. */
+ * eta_max of the C algorithm stays the rate given to ga_create (Algorithm "C Coefficient
+ * Calculation" takes the maximal rate as an input, normally the first one), so the Gap penalty
+ * relaxes as the rate decays (Section 5.1). lr must be positive and finite. */
 int ga_set_lr(ga_engine* e, float lr);
 
 /* GA_GA_LAYER only, before the first arrival: layer p is elements [offsets_host[p],
@@ -134,16 +139,17 @@ int ga_num_layers(ga_engine* e);
  * moment m_p behind C_p, n_layers floats each, into host memory (either may be NULL). */
 int ga_get_layer_state(ga_engine* e, float* gaps_host, float* m_host);
 
-/* theta <- theta0 and every worker's saved copy <- theta0 ("Initialize theta^i = theta_0",
- * Algorithm "DANA-Gap-Aware: master" line 1; the same convention is used for GA); v, m, the
- * arrival counter and iter[] are reset to 0. theta0_dev: n_params floats on the device. */
+/* theta <- theta0 and every worker's saved copy <- theta0 (the initialisation step of Algorithm
+ * "DANA-Gap-Aware: master"; the same convention is used for GA); v, m, the arrival counter and
+ * iter[] are reset to 0. theta0_dev: n_params floats on the device. */
 int ga_set_params(ga_engine* e, const float* theta0_dev);
 
-/* "Send theta to worker i" (Algorithm "Momentum-ASGD: worker": "Receive parameters"): copies the
- * master parameters into worker's saved copy with TMA bulk copies (the DANA variants compute and
- * store the estimate theta - eta gamma sum_j v^j instead), records iter[worker] <-
- * arrivals applied so far, and returns the device address of that copy (library-owned, stable for
- * the engine's life; contents change at that worker's next pull or batched push). NULL on error. */
+/* The master's send step (the worker side of it is the first step of Algorithm "Momentum-ASGD:
+ * worker"): copies the master parameters into worker's saved copy with TMA bulk copies (the DANA
+ * variants compute and store the estimate theta - eta gamma sum_j v^j instead), records
+ * iter[worker] <- arrivals applied so far, and returns the device address of that copy
+ * (library-owned, stable for the engine's life; contents change at that worker's next pull or
+ * batched push). NULL on error. */
 const float* ga_pull(ga_engine* e, int worker);
 
 /* Device address of worker's saved copy theta^worker (n_params floats) without copying anything:
@@ -158,9 +164,9 @@ const float* ga_saved(ga_engine* e, int worker);
  * without pulling; its Gap is then still measured against its last saved copy. */
 int64_t ga_push(ga_engine* e, int worker, const float* grad_dev);
 
-/* K arrivals in FIFO order (Appendix "Algorithms": "the master's scheme is a simple FIFO"),
- * each followed at once by that worker's pull -- the "Save and send current parameters" line of
- * Algorithm "Gap-Aware: master". Equivalent to { ga_push(schedule[j], grads[j]);
+/* K arrivals applied in the order given -- the master serves gradients first come, first served
+ * (Appendix "Algorithms") -- each followed at once by that worker's pull, the save-and-send step
+ * that closes Algorithm "Gap-Aware: master". Equivalent to { ga_push(schedule[j], grads[j]);
  * ga_pull(schedule[j]); } for j = 0..K-1, but up to GA_OPT_WINDOW consecutive arrivals are applied
  * by one kernel that reads and writes theta, v, m once (legal because every step is independent
  * per parameter, Section 5.3). A window is cut where a worker repeats. schedule_host: K worker
@@ -174,8 +180,9 @@ int ga_push_batch(ga_engine* e, const int* schedule_host, const float* const* gr
  * gives full PCIe speed): grads_host[j] points to n_params floats on the host; when
  * sent_out_host is not NULL, sent_out_host[j] receives the parameters sent to worker
  * schedule[j] after its arrival (n_params floats each). The parameter range is processed in
- * chunks so that host-to-device copies, the update kernel and device-to-host copies overlap.
- * Synchronous: returns when all results are in host memory. */
+ * chunks so that host-to-device copies, the update kernel and device-to-host copies overlap,
+ * across the windows of the call as well as within them. Synchronous: returns when all results
+ * are in host memory. Allocates its staging buffers (2 x 16 x 16 MiB) on first use. */
 int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* const* grads_host,
                        int K, int64_t* delays_out_host, float* const* sent_out_host);
 
@@ -193,8 +200,22 @@ int ga_gap(ga_engine* e, int worker, float* gap_out_dev);
 
 int ga_set_option(ga_engine* e, int key, double value);
 
-/* Sum and maximum over all parameters of the Gap used by the most recent GA arrival (needs
- * GA_OPT_STATS = 1 before that push). GA_ERR_STATE when none is available. */
+/* Gap statistics of every arrival of the most recent ga_push, ga_push_batch or
+ * ga_push_batch_host call, oldest first: sum_gap_host[q] and max_gap_host[q] are the sum and the
+ * maximum over all parameters of the Gap that arrival was penalised with (sum / n_params is the
+ * average Gap that Appendix "Gap and Delay" logs; Section 5.1 compares it with the delay). All
+ * windows of the call are covered, not only the last launch. Needs GA_OPT_STATS = 1 before the call
+ * and a parameter-wise Gap-Aware variant (GA_GA, GA_DANA_GA, GA_ADAM_GA), else GA_ERR_STATE. The
+ * engine keeps the last GA_STATS_LOG arrivals of a call; when the call had more, or cap is smaller,
+ * the most recent ones are returned. Both arrays hold cap doubles on the host. The sum is
+ * accumulated in fp64 in a fixed order (reproducible run to run). Synchronises the stream.
+ * Returns the number of pairs written (0 when no arrival has been applied since the option was set,
+ * ga_set_params or ga_import_state), or a negative error. */
+#define GA_STATS_LOG 4096
+int ga_get_stats_window(ga_engine* e, double* sum_gap_host, double* max_gap_host, int cap);
+
+/* The last pair of ga_get_stats_window: the Gap statistics of the most recent arrival.
+ * GA_ERR_STATE when none is available. */
 int ga_get_stats(ga_engine* e, double* sum_gap, double* max_gap);
 
 /* Arrivals applied so far, and iter[worker]. Negative on error. */

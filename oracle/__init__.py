@@ -227,3 +227,26 @@ class Oracle:
 
     def iter(self, worker):
         return int(self._l.gao_iter(self._h, worker))
+
+
+_LIB_OMP = os.path.join(_HERE, "libga_oracle_omp.so")
+
+
+def build_openmp(force=False):
+    """The same source split across threads (-fopenmp -DGAO_OPENMP): only for timing the oracle
+    on all host cores; parity always uses the single-threaded build."""
+    if not force and os.path.exists(_LIB_OMP) and os.path.getmtime(_LIB_OMP) >= os.path.getmtime(_SRC):
+        return _LIB_OMP
+    tmp = f"{_LIB_OMP}.{os.getpid()}.tmp"
+    try:
+        subprocess.check_call(["g++", *CXXFLAGS, "-fopenmp", "-DGAO_OPENMP", "-o", tmp, _SRC])
+    except OSError:
+        if os.path.exists(_LIB_OMP) and not force:
+            return _LIB_OMP
+        raise
+    os.replace(tmp, _LIB_OMP)
+    return _LIB_OMP
+
+
+def lib_openmp():
+    return _bind(build_openmp())

@@ -13,8 +13,8 @@
 //   push, variant GA   : Algorithm "Gap-Aware: master" (Section 5) with the
 //                        parameter-wise Gap of Section 5.3 (|theta_k - theta_{k-tau}|/C + 1)
 //   C                  : Algorithm "C Coefficient Calculation" (Appendix, C Coefficient)
-//   pull               : "Send theta_{k+1} to worker i" / "Save and send current
-//                        parameters" of the three master algorithms; the saved copy is
+//   pull               : the closing send step (for GA: save, then send) of the three master
+//                        algorithms; the saved copy is
 //                        the theta^i = theta_{k-tau_k} of the appendix's remark
 //   push, ADAM*        : Algorithms "Adam: master", "Adam-Staleness-Aware: master" and
 //                        "Adam-Gap-Aware: master" (appendix): the penalty (1/tau or 1/G) enters
@@ -35,7 +35,7 @@
 //     the update vector actually applied (the master's new v). 1 = "Adam order": first
 //     u = gamma v + g with the raw gradient (the printed line of the C algorithm),
 //     m <- beta m + (1-beta) u^2, C from the new m, then Gap, penalised gradient, v, theta.
-//   * "Initialize C <- 0": before any refresh, C = eta_max * eps (the last line of the C
+//   * The C algorithm starts from C = 0: before any refresh, C = eta_max * eps (the last line of the C
 //     algorithm at m_hat = 0), so the first Gap is 0/C + 1 = 1, not 0/0.
 //   * The exponent of the bias correction is the number of refreshes of m so far.
 //   * eps = 1e-8 is added after the square root, inside the eta_max product.
@@ -48,13 +48,13 @@
 //     sum, S <- (S - v^i_old) + v^i_new at each arrival (what a master would do; default);
 //     0 = the printed sum_{j=1..N} v^j evaluated afresh, in order, at every send. The two are
 //     equal in exact arithmetic and are pinned against each other.
-//   * Adam-GA's C: the C algorithm needs an "update step gamma v + g", and Adam has no momentum
+//   * Adam-GA's C: the C algorithm is written for a momentum update step gamma v + g, and Adam has no momentum
 //     coefficient, so it is run with gamma = 0: m is the running second moment of the raw
 //     gradient with the constant beta given at creation (its own state, separate from Adam's
 //     v); c_order decides as before whether the Gap sees m before or after this arrival's refresh.
 //   * Adam's bias corrections use k = the arrival index; m_hat = m * (1/(1-beta1^k)) with the
 //     reciprocal formed in double and rounded once, as for C.
-//   * Layer-wise / global C: the C algorithm "executed per layer": m_p is the running average
+//   * Layer-wise / global C: the C algorithm run once per layer: m_p is the running average
 //     of the squared NORM of layer p's update vector, C_p = eta_max (sqrt(m_p / (1 - beta^k))
 //     + eps). Squared norms are accumulated in fp64 and rounded once to the working precision
 //     (a sum of millions of fp32 terms has no meaningful fp32 order). Lagged order only.
@@ -75,6 +75,19 @@
 #include <cstring>
 #include <new>
 #include <vector>
+
+// The parity reference is this file built single-threaded. Built a second time with
+// -fopenmp -DGAO_OPENMP, the loops over parameters (independent per parameter) are split across
+// threads; that build exists only so that the benchmark can time the same program on all host
+// cores, and a test holds it to the single-threaded build bit for bit (the statistics' fp64 sum
+// changes its order, nothing else does).
+#ifdef GAO_OPENMP
+#define GAO_PARALLEL _Pragma("omp parallel for schedule(static)")
+#define GAO_PARALLEL_STATS _Pragma("omp parallel for schedule(static) reduction(+ : sum_gap) reduction(max : max_gap)")
+#else
+#define GAO_PARALLEL
+#define GAO_PARALLEL_STATS
+#endif
 
 namespace {
 
@@ -110,15 +123,15 @@ struct Master {
     int64_t k_c = 0;            // refreshes of m so far
     double last_sum_gap = 0.0, last_max_gap = 0.0;
 
-    // The gradient the master works with. Appendix "Weight Decay": under GA the gradient
-    // contains the weight-decay element, which is divided by the Gap as a part of the gradient;
-    // the master forms it from its current parameters, g + lambda * theta_k (one FMA).
+    // The gradient the master works with. Appendix "Weight Decay": under GA the decay term
+    // belongs to the gradient and is penalised by the Gap with it; the master forms it from its
+    // current parameters, g + lambda * theta_k (one FMA).
     T gw(const float* grad, int64_t j) const {
         return wd == (T)0 ? (T)grad[j] : std::fma(wd, theta[j], (T)grad[j]);
     }
 
     // The parameter step of the one-momentum-vector masters. Printed form: theta - eta v_{k+1}.
-    // Nesterov form (the paper's runs use "a NAG optimizer" but print no master-side formula;
+    // Nesterov form (Section 6 says the runs used Nesterov momentum but no master algorithm is printed that way;
     // this is the form of the common framework optimisers): theta - eta (g_hat + gamma v_{k+1}).
     T step(T th, T v_new, T g_pen, T e) const {
         if (!nesterov) return std::fma(-e, v_new, th);
@@ -203,6 +216,7 @@ struct Master {
         const T inv_bias2 = (T)(1.0 / (1.0 - std::pow((double)beta2, (double)k)));
         double sum_gap = 0.0, max_gap = 0.0;
         if (variant == ADAM_GA && c_order == 1) {
+            GAO_PARALLEL
             for (int64_t j = 0; j < d; ++j) {
                 const T g = gw(grad, j);
                 m[j] = std::fma(beta, m[j], one_minus_beta * (g * g));
@@ -210,6 +224,7 @@ struct Master {
             k_c += 1;
         }
         const T ib = k_c > 0 ? inv_bias() : (T)0;
+        GAO_PARALLEL_STATS
         for (int64_t j = 0; j < d; ++j) {
             const T g = gw(grad, j);
             T first;                                         // what is added to beta_1 m
@@ -240,13 +255,15 @@ struct Master {
 
     void pull(int i) {
         if (is_dana()) { pull_dana(i); return; }
+        GAO_PARALLEL
         for (int64_t j = 0; j < d; ++j) saved[(size_t)i * d + j] = theta[j];
         iter[i] = k_done;
     }
 
-    // DANA: "Send estimate theta_hat = theta - eta gamma sum_j v^j to worker i" (and save it).
+    // DANA's send step: the worker gets the estimate theta - eta gamma sum_j v^j, which is also saved.
     void pull_dana(int i) {
         const T eta_gamma = eta * gamma;
+        GAO_PARALLEL
         for (int64_t j = 0; j < d; ++j) {
             T total = vsum[j];
             if (dana_sum == 0) {
@@ -265,6 +282,7 @@ struct Master {
         const T one_minus_beta = (T)(1.0 - (double)beta);
         double sum_gap = 0.0, max_gap = 0.0;
         if (variant == DANA_GA && c_order == 1) {
+            GAO_PARALLEL
             for (int64_t j = 0; j < d; ++j) {
                 const T u = std::fma(gamma, vi[j], gw(grad, j));
                 m[j] = std::fma(beta, m[j], one_minus_beta * (u * u));
@@ -272,6 +290,7 @@ struct Master {
             k_c += 1;
         }
         const T ib = k_c > 0 ? inv_bias() : (T)0;
+        GAO_PARALLEL_STATS
         for (int64_t j = 0; j < d; ++j) {
             const T g = gw(grad, j);
             T g_pen = g;                                   // DANA: the gradient as it is
@@ -293,6 +312,7 @@ struct Master {
             vsum[j] = (vsum[j] - v_old) + v_new;           // running sum_j v^j
         }
         if (variant == DANA_GA && c_order == 0) {
+            GAO_PARALLEL
             for (int64_t j = 0; j < d; ++j)
                 m[j] = std::fma(beta, m[j], one_minus_beta * (vi[j] * vi[j]));
             k_c += 1;
@@ -312,12 +332,14 @@ struct Master {
         } else if (variant == GA_LAYER) {
             push_layers(i, grad);
         } else if (variant == SA_GRAD) {
+            GAO_PARALLEL
             for (int64_t j = 0; j < d; ++j) {
                 const T g_tau = gw(grad, j) / (T)tau;
                 v[j] = std::fma(gamma, v[j], g_tau);
                 theta[j] = step(theta[j], v[j], g_tau, eta);
             }
         } else if (variant == ASGD) {
+            GAO_PARALLEL
             for (int64_t j = 0; j < d; ++j) {
                 const T g = gw(grad, j);
                 v[j] = std::fma(gamma, v[j], g);
@@ -325,6 +347,7 @@ struct Master {
             }
         } else if (variant == SA) {
             const T eta_tau = eta / (T)tau;
+            GAO_PARALLEL
             for (int64_t j = 0; j < d; ++j) {
                 const T g = gw(grad, j);
                 v[j] = std::fma(gamma, v[j], g);
@@ -335,6 +358,7 @@ struct Master {
             double sum_gap = 0.0, max_gap = 0.0;
             if (c_order == 1) {
                 // Adam order: refresh m from u = gamma v + g (raw gradient) first.
+                GAO_PARALLEL
                 for (int64_t j = 0; j < d; ++j) {
                     const T u = std::fma(gamma, v[j], gw(grad, j));
                     m[j] = std::fma(beta, m[j], one_minus_beta * (u * u));
@@ -342,6 +366,7 @@ struct Master {
                 k_c += 1;
             }
             const T ib = k_c > 0 ? inv_bias() : (T)0;
+            GAO_PARALLEL_STATS
             for (int64_t j = 0; j < d; ++j) {
                 const T g = gw(grad, j);
                 const T C = coeff(m[j], ib);
@@ -355,6 +380,7 @@ struct Master {
                 if ((double)G > max_gap) max_gap = (double)G;
             }
             if (c_order == 0) {
+                GAO_PARALLEL
                 for (int64_t j = 0; j < d; ++j)
                     m[j] = std::fma(beta, m[j], one_minus_beta * (v[j] * v[j]));
                 k_c += 1;
@@ -462,7 +488,7 @@ void gao_set_c_order(void* p, int c_order) {
 }
 
 // Learning rate eta_k of the coming arrivals; eta_max of the C algorithm stays as created
-// (Appendix "C Coefficient": "usually eta_max = eta_1").
+// (the C algorithm takes the maximal rate as an input of its own, normally the first rate).
 void gao_set_lr(void* p, double lr) {
     auto* h = (Handle*)p;
     if (h->precision == 32) h->f->eta = (float)lr; else h->g->eta = (double)(float)lr;

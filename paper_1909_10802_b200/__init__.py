@@ -23,6 +23,7 @@ GA_THETA, GA_V, GA_M, GA_C, GA_V2 = 0, 1, 2, 3, 4
  GA_OPT_WEIGHT_DECAY, GA_OPT_NESTEROV) = range(8)
 GA_MAX_WINDOW = 16
 GA_NOALLOC_MAX_PARAMS = 1 << 28
+GA_STATS_LOG = 4096
 VARIANTS = {"ASGD": GA_ASGD, "SA": GA_SA, "GA": GA_GA, "SA_GRAD": GA_SA_GRAD, "DANA": GA_DANA,
             "DANA_SA": GA_DANA_SA, "DANA_GA": GA_DANA_GA, "ADAM": GA_ADAM, "ADAM_SA": GA_ADAM_SA,
             "ADAM_GA": GA_ADAM_GA, "GA_LAYER": GA_GA_LAYER}
@@ -48,6 +49,7 @@ _SIGNATURES = {
     "ga_gap": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p]),
     "ga_set_option": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_double]),
     "ga_get_stats": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
+    "ga_get_stats_window": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_int]),
     "ga_num_arrivals": (_c.c_int64, [_c.c_void_p]),
     "ga_worker_iter": (_c.c_int64, [_c.c_void_p, _c.c_int]),
     "ga_export_state": (_c.c_size_t, [_c.c_void_p, _c.c_void_p, _c.c_size_t]),
@@ -266,6 +268,12 @@ class Engine:
         s, m = ctypes.c_double(), ctypes.c_double()
         _check(self._l.ga_get_stats(self._h, ctypes.byref(s), ctypes.byref(m)))
         return s.value, m.value
+
+    def get_stats_window(self, cap=GA_STATS_LOG):
+        """[(sum of the Gap, max of the Gap)] for every arrival of the most recent push call, oldest first."""
+        s, m = (ctypes.c_double * cap)(), (ctypes.c_double * cap)()
+        n = _check(self._l.ga_get_stats_window(self._h, s, m, cap))
+        return list(zip(s[:n], m[:n]))
 
     @property
     def num_arrivals(self):

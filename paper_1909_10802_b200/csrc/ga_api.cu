@@ -31,7 +31,9 @@ int fail(int code, const char* fmt, ...) {
 
 constexpr long long kRowAlign = 32;            // floats: rows start on 128-byte boundaries
 constexpr long long kHostChunk = 4ll << 20;    // floats per chunk of the host-buffer path
+constexpr int kHostD2hRing = 4;                // chunks the kernels may run ahead of the copies out
 constexpr uint32_t kStateMagic = 0x47415331;   // "GAS1"
+constexpr int kStatsLog = GA_STATS_LOG;        // arrivals whose Gap statistics are kept
 
 }  // namespace
 
@@ -61,17 +63,20 @@ struct ga_engine {
     bool cuda_failed = false;
     // statistics
     ga::StatsPartial* partials = nullptr;
-    double* stats_dev = nullptr;   // kMaxWindow x {sum, max}
+    double* stats_dev = nullptr;   // ring of kStatsLog x {sum, max}: one pair per arrival
     int stats_blocks = 0;
-    bool stats_valid = false;
-    int stats_slot = 0;
-    // pull kernel error flag
+    int64_t stats_total = 0;       // arrivals logged since the current call began (slot = index % kStatsLog)
+    // pull kernel error flag: one int of pinned, device-mapped host memory
     int* pull_err = nullptr;
+    // beta^k, gamma^k, beta2^k carried from one arrival to the next (see inv_one_minus_pow)
+    struct PowCache { double base = 0.0, p = 0.0; int64_t k = -1; };
+    PowCache pow_c, pow_b1, pow_b2;
     // host-buffer path
     float* stage[2] = {nullptr, nullptr};
     long long stage_elems = 0;
     cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
     cudaEvent_t ev_h2d[2] = {nullptr, nullptr}, ev_kernel[2] = {nullptr, nullptr}, ev_prev = nullptr;
+    cudaEvent_t ev_d2h[kHostD2hRing] = {};
 
     float* row(int i) const { return saved + (size_t)i * stride; }
     float* vrow(int i) const { return vworker ? vworker + (size_t)i * stride : nullptr; }
@@ -95,10 +100,29 @@ struct ga_engine {
         h.nesterov = nesterov;
         return h;
     }
+    // (float)(1 / (1 - base^k)), base^k = pow(base, k) in double. Consecutive k reuse the previous
+    // power: p = p_prev * base drifts from pow() by far less than 1e-13 relative between the
+    // re-synchronisations every 64 steps, and the result is monotone in p, so whenever both
+    // ends of p (1 -+ 1e-13) round to the same float that float is also what pow() gives;
+    // otherwise pow() itself decides.
+    static float inv_one_minus_pow(PowCache& c, double base, int64_t k) {
+        if (c.k >= 0 && c.base == base && k == c.k + 1 && (k & 63) != 0) {
+            const double p = c.p * base;
+            c.p = p;
+            c.k = k;
+            const float lo = (float)(1.0 / (1.0 - p * (1.0 - 1e-13)));
+            const float hi = (float)(1.0 / (1.0 - p * (1.0 + 1e-13)));
+            if (lo == hi) return lo;
+        }
+        c.base = base;
+        c.k = k;
+        c.p = std::pow(base, (double)k);
+        return (float)(1.0 / (1.0 - c.p));
+    }
     // 1/(1-beta^k) for the C in force after k refreshes of m; 0 before the first (C = eta_max*eps)
-    float inv_bias(int64_t k) const {
+    float inv_bias(int64_t k) {
         if (k <= 0) return 0.f;
-        return (float)(1.0 / (1.0 - std::pow((double)beta, (double)k)));
+        return inv_one_minus_pow(pow_c, (double)beta, k);
     }
 };
 
@@ -142,11 +166,12 @@ int check_dev_ptr(const void* p, const char* name) {
     return GA_OK;
 }
 
-// After a synchronisation: did a bulk-copy wait of a pull kernel run out?
-int check_pull_flag(ga_engine* e) {
-    int flag = 0;
-    GA_CUDA(e, cudaMemcpy(&flag, e->pull_err, sizeof flag, cudaMemcpyDeviceToHost));
-    if (flag) {
+// Every synchronising call ends here: wait for the engine's stream, then see whether a
+// bulk-copy wait of a pull kernel ran out (the kernel raises a flag in mapped host memory). Such
+// a pull left its saved copy incomplete, so the failure is sticky like a CUDA error.
+int sync_and_check(ga_engine* e) {
+    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    if (*(volatile int*)e->pull_err) {
         e->cuda_failed = true;
         return fail(GA_ERR_CUDA, "a bulk copy of ga_pull did not complete within its wait limit");
     }
@@ -162,8 +187,11 @@ int grid_1d(long long n, int threads, int cap) {
 // ----------------------------------------------------------------------------- launch
 int launch_layer_arrival(ga_engine* e, const float* grad, float* saved_row, bool write_saved, float inv_bias);
 
+// stats_mode (STATS instantiations): 1 = the arrivals' pairs overwrite their log slots, 2 = they are
+// merged into them (a later chunk of the same arrivals on the host-buffer path)
 template <int FAMILY, int PENALTY, bool EXACT, int C_ORDER, bool STATS>
-void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st) {
+void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st,
+                     int stats_mode) {
     const long long nvec = vec_end - vec_begin;
     long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
@@ -179,15 +207,16 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
     else { if (wd) GA_LAUNCH(GA_WINDOW_BATCH, ST, true); else GA_LAUNCH(GA_WINDOW_BATCH, ST, false); }
 #undef GA_LAUNCH
     if (STATS) {
-        ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev);
+        ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev, e->stats_total,
+                                                        kStatsLog, stats_mode == 2);
     }
 }
 
 template <int FAMILY>
-void launch_family(ga_engine* e, const ga::Window& w, long long vb, long long ve, cudaStream_t st, bool stats) {
+void launch_family(ga_engine* e, const ga::Window& w, long long vb, long long ve, cudaStream_t st, int stats) {
     if (e->is_gap()) {
         const bool exact = !e->fast_math;
-#define GA_CASE(EX, CO, ST) launch_window_t<FAMILY, ga::PEN_GAP, EX, CO, ST>(e, w, vb, ve, st)
+#define GA_CASE(EX, CO, ST) launch_window_t<FAMILY, ga::PEN_GAP, EX, CO, ST>(e, w, vb, ve, st, stats)
         if (exact) {
             if (e->c_order == 0) { if (stats) GA_CASE(true, 0, true); else GA_CASE(true, 0, false); }
             else { if (stats) GA_CASE(true, 1, true); else GA_CASE(true, 1, false); }
@@ -197,14 +226,17 @@ void launch_family(ga_engine* e, const ga::Window& w, long long vb, long long ve
         }
 #undef GA_CASE
     } else if (e->is_tau_grad()) {
-        launch_window_t<FAMILY, ga::PEN_TAU, true, 0, false>(e, w, vb, ve, st);
+        launch_window_t<FAMILY, ga::PEN_TAU, true, 0, false>(e, w, vb, ve, st, 0);
     } else {
-        launch_window_t<FAMILY, ga::PEN_NONE, true, 0, false>(e, w, vb, ve, st);
+        launch_window_t<FAMILY, ga::PEN_NONE, true, 0, false>(e, w, vb, ve, st, 0);
     }
 }
 
+// One launch for arrivals w over vectors [vec_begin, vec_end). first_range / last_range say whether
+// this range is the first / last of the arrivals' parameter ranges (both true for a whole vector):
+// the Gap statistics of an arrival are complete, and counted, once its last range has run.
 int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st,
-                  bool allow_stats = true) {
+                  bool first_range = true, bool last_range = true) {
     if (vec_end <= vec_begin || w.K <= 0) return GA_OK;
     if (e->is_layer()) {   // a layer's norm needs the whole vector between arrivals: no fusion in time
         if (vec_begin != 0 || vec_end != e->stride / 4)
@@ -213,12 +245,12 @@ int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long l
             if (int rc = launch_layer_arrival(e, w.grad[j], w.saved[j], w.write_saved != 0, w.inv_bias[j])) return rc;
         return GA_OK;
     }
-    const bool stats = allow_stats && e->stats && e->is_gap();
+    const int stats = (e->stats && e->is_gap()) ? (first_range ? 1 : 2) : 0;
     if (e->is_dana()) launch_family<ga::DANA>(e, w, vec_begin, vec_end, st, stats);
     else if (e->is_adam()) launch_family<ga::ADAM>(e, w, vec_begin, vec_end, st, stats);
     else launch_family<ga::MOM>(e, w, vec_begin, vec_end, st, stats);
     GA_CUDA(e, cudaGetLastError());
-    if (stats) { e->stats_valid = true; e->stats_slot = w.K - 1; }
+    if (stats && last_range) e->stats_total += w.K;
     return GA_OK;
 }
 
@@ -298,8 +330,8 @@ void fill_window(ga_engine* e, ga::Window& w, const int* workers, const float* c
         w.tau[j] = (float)tau;
         w.bias1[j] = w.bias2[j] = 1.f;
         if (e->is_adam()) {   // Adam's bias corrections use the arrival index
-            w.bias1[j] = (float)(1.0 / (1.0 - std::pow((double)e->gamma, (double)k)));
-            w.bias2[j] = (float)(1.0 / (1.0 - std::pow((double)e->beta2, (double)k)));
+            w.bias1[j] = ga_engine::inv_one_minus_pow(e->pow_b1, (double)e->gamma, k);
+            w.bias2[j] = ga_engine::inv_one_minus_pow(e->pow_b2, (double)e->beta2, k);
         }
         w.eta_eff[j] = e->variant == GA_SA ? e->lr / (float)tau : e->lr;
         if (e->is_gap()) {
@@ -361,6 +393,7 @@ int ensure_host_path(ga_engine* e) {
         GA_CUDA(e, cudaEventCreateWithFlags(&e->ev_kernel[s], cudaEventDisableTiming));
     }
     GA_CUDA(e, cudaEventCreateWithFlags(&e->ev_prev, cudaEventDisableTiming));
+    for (int q = 0; q < kHostD2hRing; ++q) GA_CUDA(e, cudaEventCreateWithFlags(&e->ev_d2h[q], cudaEventDisableTiming));
     GA_CUDA(e, cudaStreamCreateWithFlags(&e->s_h2d, cudaStreamNonBlocking));
     GA_CUDA(e, cudaStreamCreateWithFlags(&e->s_d2h, cudaStreamNonBlocking));
     return GA_OK;
@@ -378,6 +411,10 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
     if (n_params == 0 || n_params > (size_t)1 << 34) { fail(GA_ERR_ARG, "n_params out of range"); return nullptr; }
     if (n_workers <= 0 || n_workers > 65536) { fail(GA_ERR_ARG, "n_workers out of range"); return nullptr; }
     if (!(lr > 0.f) || !std::isfinite(lr)) { fail(GA_ERR_ARG, "lr must be positive and finite"); return nullptr; }
+    if (!(lr * 1e-8f > 0.f)) {   // C = eta_max (sqrt(m_hat) + eps) must stay positive: a Gap of x/0 has no meaning
+        fail(GA_ERR_ARG, "lr is so small that lr * 1e-8 (the smallest C) rounds to zero");
+        return nullptr;
+    }
     if (!(std::fabs(momentum) < 1.f)) { fail(GA_ERR_ARG, "|momentum| must be < 1"); return nullptr; }
     if (!(c_beta >= 0.f && c_beta < 1.f)) { fail(GA_ERR_ARG, "c_beta must be in [0, 1)"); return nullptr; }
     if (variant < GA_ASGD || variant > GA_GA_LAYER) { fail(GA_ERR_ARG, "unknown variant %d", variant); return nullptr; }
@@ -406,15 +443,15 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
               cudaMalloc(&e->mom, row_bytes) == cudaSuccess &&
               cudaMalloc(&e->saved, row_bytes * (size_t)n_workers) == cudaSuccess &&
               cudaMalloc(&e->partials, sizeof(ga::StatsPartial) * (size_t)e->stats_blocks * ga::kMaxWindow) == cudaSuccess &&
-              cudaMalloc(&e->stats_dev, sizeof(double) * 2 * ga::kMaxWindow) == cudaSuccess &&
-              cudaMalloc(&e->pull_err, sizeof(int)) == cudaSuccess &&
+              cudaMalloc(&e->stats_dev, sizeof(double) * 2 * kStatsLog) == cudaSuccess &&
+              cudaHostAlloc(&e->pull_err, sizeof(int), cudaHostAllocMapped) == cudaSuccess &&
               (!e->is_dana() || cudaMalloc(&e->vworker, row_bytes * (size_t)n_workers) == cudaSuccess) &&
               (!e->is_adam() || cudaMalloc(&e->sec, row_bytes) == cudaSuccess);
     if (ok) {
         ok = cudaMemset(e->theta, 0, row_bytes) == cudaSuccess && cudaMemset(e->vel, 0, row_bytes) == cudaSuccess &&
              cudaMemset(e->mom, 0, row_bytes) == cudaSuccess &&
              cudaMemset(e->saved, 0, row_bytes * (size_t)n_workers) == cudaSuccess &&
-             cudaMemset(e->pull_err, 0, sizeof(int)) == cudaSuccess &&
+             (*e->pull_err = 0, true) &&
              (!e->vworker || cudaMemset(e->vworker, 0, row_bytes * (size_t)n_workers) == cudaSuccess) &&
              (!e->sec || cudaMemset(e->sec, 0, row_bytes) == cudaSuccess) &&
              cudaFuncSetAttribute(ga::ga_pull_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -447,13 +484,14 @@ void ga_destroy(ga_engine* e) {
     free_layers(e);
     cudaFree(e->partials);
     cudaFree(e->stats_dev);
-    cudaFree(e->pull_err);
+    cudaFreeHost(e->pull_err);
     for (int s = 0; s < 2; ++s) {
         cudaFree(e->stage[s]);
         if (e->ev_h2d[s]) cudaEventDestroy(e->ev_h2d[s]);
         if (e->ev_kernel[s]) cudaEventDestroy(e->ev_kernel[s]);
     }
     if (e->ev_prev) cudaEventDestroy(e->ev_prev);
+    for (int q = 0; q < kHostD2hRing; ++q) if (e->ev_d2h[q]) cudaEventDestroy(e->ev_d2h[q]);
     if (e->s_h2d) cudaStreamDestroy(e->s_h2d);
     if (e->s_d2h) cudaStreamDestroy(e->s_d2h);
     cudaGetLastError();
@@ -483,7 +521,7 @@ int ga_set_layers(ga_engine* e, const int64_t* offsets_host, int n_layers) {
     for (int p = 0; p < n_layers; ++p)
         if (offsets_host[p + 1] <= offsets_host[p]) return fail(GA_ERR_ARG, "layer %d is empty or out of order", p);
     DeviceGuard guard(e->device);
-    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    if (int rc = sync_and_check(e)) return rc;
     return build_layers(e, offsets_host, n_layers);
 }
 
@@ -500,8 +538,7 @@ int ga_get_layer_state(ga_engine* e, float* gaps_host, float* m_host) {
     const size_t bytes = sizeof(float) * e->n_layers();
     if (gaps_host) GA_CUDA(e, cudaMemcpyAsync(gaps_host, e->layer_gap, bytes, cudaMemcpyDeviceToHost, e->stream));
     if (m_host) GA_CUDA(e, cudaMemcpyAsync(m_host, e->m_layer, bytes, cudaMemcpyDeviceToHost, e->stream));
-    GA_CUDA(e, cudaStreamSynchronize(e->stream));
-    return GA_OK;
+    return sync_and_check(e);
 }
 
 int ga_set_params(ga_engine* e, const float* theta0_dev) {
@@ -516,7 +553,7 @@ int ga_set_params(ga_engine* e, const float* theta0_dev) {
     std::fill(e->iter.begin(), e->iter.end(), 0);
     e->k_done = 0;
     e->k_c = 0;
-    e->stats_valid = false;
+    e->stats_total = 0;
     return GA_OK;
 }
 
@@ -555,6 +592,7 @@ int64_t ga_push(ga_engine* e, int worker, const float* grad_dev) {
     DeviceGuard guard(e->device);
     ga::Window w;
     int64_t tau = 0;
+    e->stats_total = 0;
     fill_window(e, w, &worker, &grad_dev, 1, /*with_pull=*/false, &tau);
     if (int rc = launch_window(e, w, 0, e->stride / 4, e->stream)) return rc;
     return tau;
@@ -566,6 +604,7 @@ int ga_push_batch(ga_engine* e, const int* schedule_host, const float* const* gr
     if (int rc = validate_batch(e, schedule_host, (const void* const*)grads_host, K, true)) return rc;
     DeviceGuard guard(e->device);
     int launches = 0;
+    if (K > 0) e->stats_total = 0;
     for (int pos = 0; pos < K;) {
         const int n = next_window(schedule_host, pos, K, e->window);
         ga::Window w;
@@ -589,23 +628,29 @@ int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* cons
     DeviceGuard guard(e->device);
     if (int rc = ensure_host_path(e)) return rc;
     int launches = 0;
+    if (K > 0) e->stats_total = 0;
     const long long chunk = e->stage_elems;
+    const long long n_chunks = (e->stride + chunk - 1) / chunk;
+    // How far the update kernels may run ahead of the copies back to the host. The kernel of
+    // window w+1 on chunk c may rewrite a saved row that the copy-out of (w, c) still reads; copies
+    // out run in order on one stream, so waiting for the copy-out issued `lag` chunks ago covers it.
+    const long long lag = n_chunks < kHostD2hRing ? n_chunks : kHostD2hRing;
     // the copy streams start after everything already enqueued on the engine's stream
     GA_CUDA(e, cudaEventRecord(e->ev_prev, e->stream));
     GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_prev, 0));
     GA_CUDA(e, cudaStreamWaitEvent(e->s_d2h, e->ev_prev, 0));
+    long long g = 0;   // chunks issued in this call, over all windows: nothing below waits on the host
     for (int pos = 0; pos < K;) {
         const int n = next_window(schedule_host, pos, K, e->window);
         ga::Window w;
         const float* staged[ga::kMaxWindow] = {};
         fill_window(e, w, schedule_host + pos, staged, n, true, delays_out_host ? delays_out_host + pos : nullptr);
-        long long c_index = 0;
-        for (long long c0 = 0; c0 < e->stride; c0 += chunk, ++c_index) {
-            const int s = (int)(c_index & 1);
+        for (long long c0 = 0, c = 0; c0 < e->stride; c0 += chunk, ++c, ++g) {
+            const int s = (int)(g & 1);
             const long long c1 = c0 + chunk < e->stride ? c0 + chunk : e->stride;
             const long long valid = (c1 < e->d ? c1 : e->d) - c0;   // floats the caller's buffers hold
-            // staging buffer s is free once the kernel of chunk c_index-2 has run
-            if (c_index >= 2) GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_kernel[s], 0));
+            // staging buffer s is free once the kernel that read it two chunks ago has run
+            if (g >= 2) GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_kernel[s], 0));
             for (int j = 0; j < n; ++j) {
                 float* dst = e->stage[s] + (size_t)j * chunk;
                 if (valid > 0)
@@ -615,24 +660,26 @@ int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* cons
             }
             GA_CUDA(e, cudaEventRecord(e->ev_h2d[s], e->s_h2d));
             GA_CUDA(e, cudaStreamWaitEvent(e->stream, e->ev_h2d[s], 0));
+            if (sent_out_host && g >= lag)
+                GA_CUDA(e, cudaStreamWaitEvent(e->stream, e->ev_d2h[(g - lag) % kHostD2hRing], 0));
             w.grad_offset = c0;
-            if (int rc = launch_window(e, w, c0 / 4, c1 / 4, e->stream, /*allow_stats=*/false)) return rc;
+            if (int rc = launch_window(e, w, c0 / 4, c1 / 4, e->stream, /*first_range=*/c == 0, /*last_range=*/c1 == e->stride))
+                return rc;
             ++launches;
             GA_CUDA(e, cudaEventRecord(e->ev_kernel[s], e->stream));
-            if (sent_out_host && valid > 0) {
+            if (sent_out_host) {
                 GA_CUDA(e, cudaStreamWaitEvent(e->s_d2h, e->ev_kernel[s], 0));
-                for (int j = 0; j < n; ++j)
+                for (int j = 0; j < n && valid > 0; ++j)
                     GA_CUDA(e, cudaMemcpyAsync(sent_out_host[pos + j] + c0, e->row(schedule_host[pos + j]) + c0,
                                                sizeof(float) * (size_t)valid, cudaMemcpyDeviceToHost, e->s_d2h));
+                GA_CUDA(e, cudaEventRecord(e->ev_d2h[g % kHostD2hRing], e->s_d2h));
             }
         }
-        // a later window may rewrite the rows being read back and reuse the staging buffers
-        GA_CUDA(e, cudaStreamSynchronize(e->s_h2d));
-        GA_CUDA(e, cudaStreamSynchronize(e->stream));
-        GA_CUDA(e, cudaStreamSynchronize(e->s_d2h));
         pos += n;
     }
-    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    GA_CUDA(e, cudaStreamSynchronize(e->s_h2d));
+    GA_CUDA(e, cudaStreamSynchronize(e->s_d2h));
+    if (int rc = sync_and_check(e)) return rc;
     return launches;
 }
 
@@ -656,8 +703,7 @@ int ga_get(ga_engine* e, int which, float* out_dev) {
     } else {
         return fail(GA_ERR_ARG, "unknown vector %d", which);
     }
-    GA_CUDA(e, cudaStreamSynchronize(e->stream));
-    return check_pull_flag(e);
+    return sync_and_check(e);
 }
 
 int ga_get_worker_momentum(ga_engine* e, int worker, float* out_dev) {
@@ -667,8 +713,7 @@ int ga_get_worker_momentum(ga_engine* e, int worker, float* out_dev) {
     if (!e->is_dana()) return fail(GA_ERR_STATE, "only the DANA variants keep a momentum vector per worker");
     DeviceGuard guard(e->device);
     GA_CUDA(e, cudaMemcpyAsync(out_dev, e->vrow(worker), sizeof(float) * (size_t)e->d, cudaMemcpyDeviceToDevice, e->stream));
-    GA_CUDA(e, cudaStreamSynchronize(e->stream));
-    return GA_OK;
+    return sync_and_check(e);
 }
 
 int ga_gap(ga_engine* e, int worker, float* gap_out_dev) {
@@ -680,8 +725,7 @@ int ga_gap(ga_engine* e, int worker, float* gap_out_dev) {
     ga::ga_gap_kernel<<<grid_1d(e->d, 256, 148 * 8), 256, 0, e->stream>>>(
         e->theta, e->row(worker), e->mom, e->inv_bias(e->k_c), e->hyper(), e->d, gap_out_dev);
     GA_CUDA(e, cudaGetLastError());
-    GA_CUDA(e, cudaStreamSynchronize(e->stream));
-    return GA_OK;
+    return sync_and_check(e);
 }
 
 int ga_set_option(ga_engine* e, int key, double value) {
@@ -701,7 +745,7 @@ int ga_set_option(ga_engine* e, int key, double value) {
         case GA_OPT_STATS:
             if (v != 0 && v != 1) return fail(GA_ERR_ARG, "GA_OPT_STATS must be 0 or 1");
             e->stats = v;
-            if (!v) e->stats_valid = false;
+            if (!v) e->stats_total = 0;
             return GA_OK;
         case GA_OPT_ADAM_BETA2:
             if (!(value >= 0.0 && value < 1.0)) return fail(GA_ERR_ARG, "GA_OPT_ADAM_BETA2 must be in [0, 1)");
@@ -709,7 +753,8 @@ int ga_set_option(ga_engine* e, int key, double value) {
             e->beta2 = (float)value;
             return GA_OK;
         case GA_OPT_ADAM_EPS:
-            if (!(value > 0.0)) return fail(GA_ERR_ARG, "GA_OPT_ADAM_EPS must be positive");
+            if (!((float)value > 0.f) || !std::isfinite((float)value))
+                return fail(GA_ERR_ARG, "GA_OPT_ADAM_EPS must be positive and finite as a float");
             if (e->k_done != 0) return fail(GA_ERR_STATE, "GA_OPT_ADAM_EPS can only change before the first arrival");
             e->adam_eps = (float)value;
             return GA_OK;
@@ -732,17 +777,32 @@ int ga_set_option(ga_engine* e, int key, double value) {
     }
 }
 
+int ga_get_stats_window(ga_engine* e, double* sum_gap_host, double* max_gap_host, int cap) {
+    if (int rc = check_engine(e)) return rc;
+    if (cap < 0 || (cap > 0 && (!sum_gap_host || !max_gap_host))) return fail(GA_ERR_ARG, "bad output arrays");
+    if (!e->stats || !e->is_gap() || e->is_layer())
+        return fail(GA_ERR_STATE, "no Gap statistics: set GA_OPT_STATS on a parameter-wise Gap-Aware variant first");
+    const int64_t kept = e->stats_total < kStatsLog ? e->stats_total : kStatsLog;
+    const int n = (int)(kept < cap ? kept : cap);
+    if (n == 0) return 0;
+    DeviceGuard guard(e->device);
+    std::vector<double> host(2 * (size_t)kStatsLog);
+    GA_CUDA(e, cudaMemcpyAsync(host.data(), e->stats_dev, sizeof(double) * host.size(), cudaMemcpyDeviceToHost, e->stream));
+    if (int rc = sync_and_check(e)) return rc;
+    for (int q = 0; q < n; ++q) {
+        const int64_t slot = (e->stats_total - n + q) % kStatsLog;
+        sum_gap_host[q] = host[2 * slot];
+        max_gap_host[q] = host[2 * slot + 1];
+    }
+    return n;
+}
+
 int ga_get_stats(ga_engine* e, double* sum_gap, double* max_gap) {
     if (int rc = check_engine(e)) return rc;
     if (!sum_gap || !max_gap) return fail(GA_ERR_ARG, "output pointer is NULL");
-    if (!e->stats_valid) return fail(GA_ERR_STATE, "no Gap statistics: enable GA_OPT_STATS before a GA push");
-    DeviceGuard guard(e->device);
-    double host[2 * ga::kMaxWindow];
-    GA_CUDA(e, cudaMemcpyAsync(host, e->stats_dev, sizeof host, cudaMemcpyDeviceToHost, e->stream));
-    GA_CUDA(e, cudaStreamSynchronize(e->stream));
-    *sum_gap = host[2 * e->stats_slot];
-    *max_gap = host[2 * e->stats_slot + 1];
-    return GA_OK;
+    if (e->stats_total == 0) return fail(GA_ERR_STATE, "no Gap statistics: enable GA_OPT_STATS before a GA push");
+    const int n = ga_get_stats_window(e, sum_gap, max_gap, 1);
+    return n == 1 ? GA_OK : (n < 0 ? n : fail(GA_ERR_STATE, "no Gap statistics available"));
 }
 
 int64_t ga_num_arrivals(ga_engine* e) {
@@ -797,8 +857,8 @@ size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap) {
         std::memcpy(p, e->layer_off.data(), sizeof(int64_t) * (n + 1)); p += sizeof(int64_t) * (n + 1);
         err = cudaMemcpyAsync(p, e->m_layer, sizeof(float) * n, cudaMemcpyDeviceToHost, e->stream);
     }
-    if (err == cudaSuccess) err = cudaStreamSynchronize(e->stream);
     if (err != cudaSuccess) { cuda_fail(e, err, "ga_export_state"); return 0; }
+    if (sync_and_check(e) != GA_OK) return 0;
     return need;
 }
 
@@ -823,12 +883,33 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
         if (n < 1 || n > (1 << 20) || len < base + sizeof(int64_t) * (n + 2) + sizeof(float) * n)
             return fail(GA_ERR_ARG, "state buffer truncated");
     } else if (len < need) return fail(GA_ERR_ARG, "state buffer truncated");
-    if ( h.window < 1 || h.window > GA_MAX_WINDOW || h.k_done < 0 || h.k_c < 0)
+    // everything a later push relies on is checked before any device state is touched
+    auto flag = [](int32_t v) { return v == 0 || v == 1; };
+    auto unit = [](float v) { return v >= 0.f && v < 1.f; };
+    if (h.window < 1 || h.window > GA_MAX_WINDOW || h.k_done < 0 || h.k_c < 0 || h.k_c > h.k_done ||
+        !flag(h.c_order) || !flag(h.fast_math) || !flag(h.stats) || !flag(h.nesterov) ||
+        !(h.lr > 0.f) || !std::isfinite(h.lr) || !(h.lr_max > 0.f) || !std::isfinite(h.lr_max) ||
+        !(h.lr_max * h.eps > 0.f) || !(h.eps > 0.f) || !std::isfinite(h.eps) || !(std::fabs(h.gamma) < 1.f) ||
+        !unit(h.beta) || !unit(h.beta2) || !(h.adam_eps > 0.f) || !std::isfinite(h.adam_eps) ||
+        !(h.weight_decay >= 0.f) || !std::isfinite(h.weight_decay) ||
+        (h.c_order == 1 && e->is_layer()) || (h.nesterov == 1 && (e->is_dana() || e->is_adam())))
         return fail(GA_ERR_ARG, "state header holds invalid values");
-    DeviceGuard guard(e->device);
     const char* p = (const char*)buf_host + sizeof h;
     std::vector<int64_t> iter(e->n_workers);
     std::memcpy(iter.data(), p, sizeof(int64_t) * e->n_workers); p += sizeof(int64_t) * e->n_workers;
+    for (int i = 0; i < e->n_workers; ++i)   // a pull cannot lie in the future: every delay stays >= 1
+        if (iter[i] < 0 || iter[i] > h.k_done)
+            return fail(GA_ERR_ARG, "state holds iter[%d] = %lld outside [0, %lld]", i, (long long)iter[i], (long long)h.k_done);
+    if (e->is_layer()) {   // the layer table too, before anything is copied
+        const char* q = (const char*)buf_host + sizeof(StateHeader) + sizeof(int64_t) * e->n_workers + vec * rows;
+        int64_t n = 0;
+        std::memcpy(&n, q, sizeof n); q += sizeof n;
+        std::vector<int64_t> off(n + 1);
+        std::memcpy(off.data(), q, sizeof(int64_t) * (n + 1));
+        if (off[0] != 0 || off[n] != e->d) return fail(GA_ERR_ARG, "state holds a layer table for another vector");
+        for (int64_t t = 0; t < n; ++t) if (off[t + 1] <= off[t]) return fail(GA_ERR_ARG, "state holds a bad layer table");
+    }
+    DeviceGuard guard(e->device);
     float* vecs[3] = {e->theta, e->vel, e->mom};
     for (int q = 0; q < 3; ++q, p += vec)
         GA_CUDA(e, cudaMemcpyAsync(vecs[q], p, vec, cudaMemcpyHostToDevice, e->stream));
@@ -842,18 +923,16 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
         std::memcpy(&n, p, sizeof n); p += sizeof n;
         std::vector<int64_t> off(n + 1);
         std::memcpy(off.data(), p, sizeof(int64_t) * (n + 1)); p += sizeof(int64_t) * (n + 1);
-        if (off[0] != 0 || off[n] != e->d) return fail(GA_ERR_ARG, "state holds a layer table for another vector");
-        for (int64_t q = 0; q < n; ++q) if (off[q + 1] <= off[q]) return fail(GA_ERR_ARG, "state holds a bad layer table");
         if (int rc = build_layers(e, off.data(), (int)n)) return rc;
         GA_CUDA(e, cudaMemcpyAsync(e->m_layer, p, sizeof(float) * n, cudaMemcpyHostToDevice, e->stream));
     }
-    GA_CUDA(e, cudaStreamSynchronize(e->stream));
+    if (int rc = sync_and_check(e)) return rc;
     e->iter = iter;
     e->k_done = h.k_done; e->k_c = h.k_c;
     e->lr = h.lr; e->gamma = h.gamma; e->beta = h.beta; e->eps = h.eps;
     e->beta2 = h.beta2; e->adam_eps = h.adam_eps; e->lr_max = h.lr_max; e->weight_decay = h.weight_decay;
     e->c_order = h.c_order; e->fast_math = h.fast_math; e->stats = h.stats; e->window = h.window; e->nesterov = h.nesterov;
-    e->stats_valid = false;
+    e->stats_total = 0;
     return GA_OK;
 }
 
@@ -963,7 +1042,7 @@ extern "C" int ga_gap_stats_noalloc(const float* theta_dev, const float* saved_d
     const int blocks = (int)((n_params + kNoAllocTile - 1) / kNoAllocTile);
     cudaStream_t st = (cudaStream_t)cuda_stream;
     ga_gap_stats_tile_kernel<<<blocks, 256, 0, st>>>(theta_dev, saved_dev, m_dev, inv_bias, h, (long long)n_params, scratch);
-    ga::ga_stats_finish_kernel<<<1, 256, 0, st>>>(scratch, blocks, out_dev);
+    ga::ga_stats_finish_kernel<<<1, 256, 0, st>>>(scratch, blocks, out_dev, 0, 1, 0);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return fail(GA_ERR_CUDA, "ga_gap_stats_noalloc launch: %s", cudaGetErrorString(err));
     return GA_OK;

@@ -1,0 +1,361 @@
+"""More parity cases through the C ABI: Gap statistics of every arrival of a call (all three
+parameter-wise Gap-Aware masters, fused windows, the host-buffer path, range shards), the
+host-buffer path for the DANA and Adam masters, DANA-GA's fast-math form, the shared-memory ring
+against the register path over a whole ResNet-50-sized vector, and what ga_import_state and
+ga_create must refuse.
+"""
+import ctypes
+import struct
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as W
+from tests.oracle_run import run_oracle, within, worst
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5     # max |gpu - ref| <= TOL * (1 + |ref|)
+GAP_VARIANTS = ["GA", "DANA_GA", "ADAM_GA"]
+
+
+@pytest.fixture(scope="module")
+def P():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_1909_10802_b200 as pkg
+    pkg.lib()
+    W.cuda_lib()
+    return pkg
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+def _oracle_stats(wl, variant, c_order=0, n_arrivals=None):
+    """(sum of the Gap, max of the Gap) of every arrival, from the oracle, and the oracle itself."""
+    o = oracle.Oracle(wl.d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, oracle.VARIANTS[variant], c_order=c_order)
+    o.set_params(wl.theta0())
+    pairs, delays = [], []
+    sched = wl.schedule()[:n_arrivals]
+    for k, i in enumerate(sched, start=1):
+        delays.append(o.push(i, wl.grad(k, o.sent_f32(i))))
+        pairs.append(o.stats())
+        o.pull(i)
+    return pairs, delays, o
+
+
+# ----------------------------------------------------------------------------- Gap statistics
+@pytest.mark.parametrize("variant", GAP_VARIANTS)
+@pytest.mark.parametrize("c_order", [0, 1])
+def test_stats_of_every_arrival_of_a_call(P, variant, c_order):
+    """Appendix "Gap and Delay" logs the average Gap over all updates: through the whole mini
+    schedule (60 arrivals, a dozen fused windows) every arrival's sum and max of the Gap must come
+    back, not only those of a window's last arrival."""
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("mini")
+    want, odelays, o = _oracle_stats(wl, variant, c_order)
+    run = Run(wl, variant, 16, options={P.GA_OPT_C_ORDER: c_order, P.GA_OPT_STATS: 1})
+    assert run.engine.get_stats_window() == []                      # nothing applied yet
+    wins = W.windows(wl.schedule(), 16)
+    got = []
+    for win in wins:                          # gradients need the copies sent so far: one window per call
+        run.step(win)
+        got += run.engine.get_stats_window()
+    assert run.delays == odelays and len(got) == len(want) == wl.arrivals
+    for k, ((s, m), (os_, om)) in enumerate(zip(got, want)):
+        assert abs(s - os_) <= 1e-9 * os_ and m == om, (variant, k, s, os_, m, om)
+    assert run.engine.get_stats() == got[-1]
+    assert len(run.engine.get_stats_window(cap=2)) == min(2, len(wins[-1]))
+    run.close()
+
+
+@pytest.mark.parametrize("variant", GAP_VARIANTS)
+def test_stats_of_a_multi_window_call(P, variant):
+    """One call whose schedule splits into three launches (a worker repeats twice): the log must
+    hold all eight arrivals in order. Gradients are fixed vectors here, so the whole schedule can
+    go into one ga_push_batch."""
+    import torch
+    d, n = 70_001, 3
+    rng = np.random.default_rng(17)
+    th0 = rng.normal(size=d).astype(np.float32)
+    sched = [0, 1, 2, 1, 0, 2, 2, 1]
+    grads = [rng.normal(size=d).astype(np.float32) for _ in sched]
+    var = oracle.VARIANTS[variant]
+    lr = 0.01 if variant == "ADAM_GA" else 0.1
+    o = oracle.Oracle(d, n, lr, 0.9, 0.999, var)
+    o.set_params(th0)
+    eng = P.Engine(d, n, lr, 0.9, 0.999, var)
+    eng.set_option(P.GA_OPT_STATS, 1)
+    eng.set_params(torch.from_numpy(th0).cuda())
+    want = []
+    for i, g in zip(sched, grads):
+        o.push(i, g)
+        want.append(o.stats())
+        o.pull(i)
+    delays, launches = eng.push_batch(sched, [torch.from_numpy(g).cuda() for g in grads], return_launches=True)
+    assert launches == len(W.windows(sched, 16)) == 3
+    got = eng.get_stats_window()
+    assert len(got) == len(sched)
+    for (s, m), (os_, om) in zip(got, want):
+        assert abs(s - os_) <= 1e-9 * os_ and m == om
+    # a single push is a call of one arrival
+    g = rng.normal(size=d).astype(np.float32)
+    eng.push(1, torch.from_numpy(g).cuda())
+    o.push(1, g)
+    (s, m), = eng.get_stats_window()
+    assert abs(s - o.stats()[0]) <= 1e-9 * o.stats()[0] and m == o.stats()[1]
+    # switched off: nothing to read
+    eng.set_option(P.GA_OPT_STATS, 0)
+    with pytest.raises(P.GaError):
+        eng.get_stats_window()
+    eng.close()
+    plain = P.Engine(64, 2, 0.1, 0.9, 0.999, P.GA_SA)
+    plain.set_option(P.GA_OPT_STATS, 1)
+    with pytest.raises(P.GaError):
+        plain.get_stats_window()
+    plain.close()
+
+
+def test_stats_log_keeps_the_most_recent_arrivals(P):
+    """A call longer than the log (GA_STATS_LOG arrivals): the newest entries survive, in order."""
+    import torch
+    d, n = 257, 2
+    rng = np.random.default_rng(2)
+    eng = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA)
+    eng.set_option(P.GA_OPT_STATS, 1)
+    th0 = rng.normal(size=d).astype(np.float32)
+    eng.set_params(torch.from_numpy(th0).cuda())
+    o = oracle.Oracle(d, n, 0.1, 0.9, 0.999, oracle.GA)
+    o.set_params(th0)
+    g = (0.01 * rng.normal(size=d)).astype(np.float32)
+    gd = torch.from_numpy(g).cuda()
+    K = P.GA_STATS_LOG + 37
+    sched = [k % n for k in range(K)]
+    want = []
+    for i in sched:
+        o.push(i, g)
+        want.append(o.stats())
+        o.pull(i)
+    eng.push_batch(sched, [gd] * K)
+    got = eng.get_stats_window()
+    assert len(got) == P.GA_STATS_LOG
+    for (s, m), (os_, om) in zip(got, want[-P.GA_STATS_LOG:]):
+        assert abs(s - os_) <= 1e-9 * os_ and m == om
+    eng.close()
+
+
+def test_stats_of_range_shards_combine_to_the_whole(P):
+    """Three engines that each own a 128-byte aligned range of the vector: the sum of their sums
+    and the maximum of their maxima are the whole engine's statistics (what
+    shard.combine_gap_stats computes with two all-reduces)."""
+    from paper_1909_10802_b200.runner import Run
+    from paper_1909_10802_b200.shard import shard_range
+    wl = W.config("mini")
+    opts = {P.GA_OPT_STATS: 1}
+    whole = Run(wl, "GA", 16, options=opts)
+    wins = W.windows(wl.schedule(), 16)
+    parts = [Run(wl, "GA", 16, options=opts, shard=shard_range(wl.d, r, 3)) for r in range(3)]
+    for win in wins:
+        whole.step(win)
+        ref = whole.engine.get_stats_window()
+        shards = []
+        for part in parts:
+            part.step(win)
+            shards.append(part.engine.get_stats_window())
+        for k, (s, m) in enumerate(ref):
+            assert abs(sum(sh[k][0] for sh in shards) - s) <= 1e-12 * s
+            assert max(sh[k][1] for sh in shards) == m
+    for r in parts + [whole]:
+        r.close()
+
+
+def test_mean_gap_below_mean_delay_on_resnet50_shape(P):
+    """Section 5.1 (soft check, on the GPU and over ALL 25.5M parameters): the average Gap stays
+    above 1 and below the average delay."""
+    import torch
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("C3")
+    run = Run(wl, "GA", 16, options={P.GA_OPT_STATS: 1})
+    gaps = []
+    for win in W.windows(wl.schedule()[:320], 16):
+        run.step(win)
+        gaps += [s / wl.d for s, _ in run.engine.get_stats_window()]
+    taus = run.delays
+    assert len(gaps) == len(taus) == 320 and min(gaps) >= 1.0
+    assert 1.0 < np.mean(gaps[160:]) < np.mean(taus[160:])
+    run.close()
+    torch.cuda.empty_cache()
+
+
+# ----------------------------------------------------------------------------- host-buffer path
+@pytest.mark.parametrize("variant", ["GA", "DANA_GA", "ADAM_GA", "DANA", "SA"])
+def test_host_buffer_path_all_families(P, variant):
+    """ga_push_batch_host on three chunks with a ragged end, two windows in one call (worker 0
+    repeats), against the device path arrival by arrival: state, sent parameters, delays and the
+    Gap statistics (merged chunk by chunk) must agree."""
+    import torch
+    d, n = 9_000_011, 3
+    rng = np.random.default_rng(3)
+    th0 = torch.from_numpy(rng.normal(size=d).astype(np.float32)).cuda()
+    sched = [2, 0, 1, 0, 2]
+    grads = [torch.from_numpy((0.1 * rng.normal(size=d)).astype(np.float32)).pin_memory() for _ in sched]
+    outs = [torch.empty(d, dtype=torch.float32).pin_memory() for _ in sched]
+    var = P.VARIANTS[variant]
+    lr = 0.01 if variant == "ADAM_GA" else 0.1
+    a = P.Engine(d, n, lr, 0.9, 0.999, var)
+    b = P.Engine(d, n, lr, 0.9, 0.999, var)
+    gap = variant in GAP_VARIANTS
+    for e_ in (a, b):
+        e_.set_params(th0)
+        if gap:
+            e_.set_option(P.GA_OPT_STATS, 1)
+    da, launches = a.push_batch_host(sched, grads, outs)
+    assert launches == 2 * 3
+    sent_dev, db, stats_b = [], [], []
+    for i, g in zip(sched, grads):
+        db += b.push_batch([i], [g.cuda()])
+        sent_dev.append(b.saved(i).clone())
+        if gap:
+            stats_b += b.get_stats_window()
+    assert da == db
+    vectors = [P.GA_THETA, P.GA_V] + ([P.GA_M] if gap else []) + ([P.GA_V2] if variant.startswith("ADAM") else [])
+    for which in vectors:
+        assert torch.equal(a.get(which), b.get(which)), which
+    if variant.startswith("DANA"):
+        for i in range(n):
+            assert torch.equal(a.get_worker_momentum(i), b.get_worker_momentum(i))
+    for o_host, s_dev in zip(outs, sent_dev):
+        assert torch.equal(o_host.cuda(), s_dev)
+    if gap:
+        stats_a = a.get_stats_window()
+        assert len(stats_a) == len(stats_b) == len(sched)
+        for (s, m), (sb, mb) in zip(stats_a, stats_b):
+            assert abs(s - sb) <= 1e-12 * sb and m == mb
+    # without result buffers (nothing is copied back) the state still advances identically
+    a.push_batch_host([1, 2], grads[:2], None)
+    b.push_batch([1, 2], [g.cuda() for g in grads[:2]])
+    assert torch.equal(a.get(P.GA_THETA), b.get(P.GA_THETA))
+    a.close()
+    b.close()
+
+
+# ----------------------------------------------------------------------------- ring path vs register path
+def test_c3_ring_path_equals_register_path_everywhere(P):
+    """ResNet-50 shape, 64 workers: after the same 208 arrivals the K = 16 launches (shared-memory
+    ring) and the K = 1 launches (register loads) must leave every element of theta, v, m and of
+    two saved copies identical -- all 200k blocks, not a sample."""
+    import torch
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("C3")
+    keep = None
+    for window in (16, 1):
+        run = Run(wl, "GA", window)
+        run.run(208)
+        last = run.wl.schedule()[207]
+        vecs = [run.engine.get(w) for w in (P.GA_THETA, P.GA_V, P.GA_M)]
+        vecs += [run.engine.saved(last).clone(), run.engine.saved(wl.schedule()[100]).clone()]
+        delays = list(run.delays)
+        run.close()
+        torch.cuda.empty_cache()
+        if keep is None:
+            keep = (vecs, delays)
+        else:
+            assert delays == keep[1]
+            for q, (x, y) in enumerate(zip(keep[0], vecs)):
+                assert torch.equal(x, y), f"vector {q} differs between K = 16 and K = 1"
+
+
+# ----------------------------------------------------------------------------- fast math, DANA-GA
+def test_dana_ga_fast_math_single_arrival(P):
+    """DANA-GA's fast form (GA_OPT_MATH = 1) against the fp64 oracle, one arrival from an
+    identical fp32 state, at the start and deep into a run."""
+    import torch
+    wl = W.Workload(name="danafast", segments=[30_000], n_workers=4, arrivals=40, schedule_kind="ticks", seed=123)
+    sched = wl.schedule()
+    for start in (0, 25):
+        o32, _, _ = run_oracle(wl, "DANA_GA", n_arrivals=start)
+        state = o32.state()
+        o64 = oracle.Oracle(wl.d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, oracle.DANA_GA, precision=64)
+        o64.set_state(*state[:7], v_workers=state[7])
+        eng = P.Engine(wl.d, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, P.GA_DANA_GA)
+        eng.set_option(P.GA_OPT_MATH, 1)
+        st = P.unpack_state(eng.export_state())
+        st.update(theta=state[0], v=state[1], m=state[2], saved=state[3], iter=state[4], k_done=state[5],
+                  k_c=state[6], v_workers=state[7])
+        eng.import_state(P.pack_state(st))
+        i = sched[start]
+        g = wl.grad(start + 1, o32.sent_f32(i))
+        assert eng.push_batch([i], [torch.from_numpy(g).cuda()]) == [o64.push(i, g)]
+        o64.pull(i)
+        pairs = [(eng.get(P.GA_THETA), o64.get(o64.THETA)), (eng.get(P.GA_V), o64.get(o64.V)),
+                 (eng.get(P.GA_M), o64.get(o64.M)), (eng.get_worker_momentum(i), o64.worker_momentum(i)),
+                 (eng.saved(i), o64.saved(i))]
+        for q, (got, ref) in enumerate(pairs):
+            assert within(_np(got), ref, TOL), (start, q, worst(_np(got), ref))
+        eng.close()
+
+
+# ----------------------------------------------------------------------------- what must be refused
+def test_lr_too_small_for_c_is_refused(P):
+    """C = eta_max (sqrt(m_hat) + 1e-8) must stay positive: a rate for which eta_max * 1e-8 rounds
+    to zero would make the Gap 0/0, so ga_create refuses it; the smallest accepted rates work."""
+    import torch
+    l = P.lib()
+    assert not l.ga_create(16, 2, 1e-38, 0.9, 0.999, P.GA_GA) and "rounds to zero" in P.last_error()
+    eng = P.Engine(1000, 2, 2e-37, 0.9, 0.999, P.GA_GA)        # eta_max * 1e-8 is a subnormal, still > 0
+    o = oracle.Oracle(1000, 2, 2e-37, 0.9, 0.999, oracle.GA)
+    rng = np.random.default_rng(4)
+    th0 = rng.normal(size=1000).astype(np.float32)
+    eng.set_params(torch.from_numpy(th0).cuda())
+    o.set_params(th0)
+    for i in (0, 1, 0):
+        g = rng.normal(size=1000).astype(np.float32)
+        assert eng.push_batch([i], [torch.from_numpy(g).cuda()]) == o.push_batch([i], [g])
+    for which, ow in ((P.GA_THETA, o.THETA), (P.GA_V, o.V), (P.GA_M, o.M), (P.GA_C, o.C)):
+        got, ref = _np(eng.get(which)), o.get(ow).astype(np.float32)
+        assert np.array_equal(got, ref, equal_nan=True), which
+    assert l.ga_set_option(eng._h, P.GA_OPT_ADAM_EPS, 1e-60) == P.GA_ERR_ARG    # zero as a float
+    eng.close()
+
+
+def test_import_state_refuses_inconsistent_headers(P):
+    """Every header field and iter[] entry that a later push relies on is checked before device
+    state is touched: a doctored checkpoint comes back as GA_ERR_ARG and the engine continues
+    exactly as if the call had not been made."""
+    import torch
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("mini")
+    a = Run(wl, "GA", 4)
+    b = Run(wl, "GA", 4)
+    a.run(30)
+    b.run(30)
+    blob = a.engine.export_state()
+    fmt = "<IIqqqqffffiiiiiiffff"
+    names = ("magic version d n_workers k_done k_c lr gamma beta eps variant c_order fast_math stats window nesterov "
+             "beta2 adam_eps lr_max weight_decay").split()
+    head = list(struct.unpack_from(fmt, blob, 0))
+    hs = struct.calcsize(fmt)
+    bad_values = {"k_done": -1, "k_c": 31, "lr": 0.0, "gamma": 1.5, "beta": 1.0, "eps": 0.0, "c_order": 2,
+                  "fast_math": -1, "stats": 7, "window": 0, "nesterov": 3, "beta2": -0.1, "adam_eps": 0.0,
+                  "lr_max": float("inf"), "weight_decay": -1.0, "variant": P.GA_SA, "d": wl.d + 1, "magic": 1}
+    for name, value in bad_values.items():
+        h = list(head)
+        h[names.index(name)] = value
+        doctored = struct.pack(fmt, *h) + blob[hs:]
+        assert a.engine._l.ga_import_state(a.engine._h, doctored, len(doctored)) == P.GA_ERR_ARG, name
+    for worker, value in ((0, 31), (2, -1)):      # a pull in the future would give a delay <= 0
+        iters = np.frombuffer(blob, dtype=np.int64, count=wl.n_workers, offset=hs).copy()
+        iters[worker] = value
+        doctored = blob[:hs] + iters.tobytes() + blob[hs + 8 * wl.n_workers:]
+        assert a.engine._l.ga_import_state(a.engine._h, doctored, len(doctored)) == P.GA_ERR_ARG
+        assert "iter" in P.last_error()
+    a.run()
+    b.run()
+    for which in (P.GA_THETA, P.GA_V, P.GA_M):
+        assert torch.equal(a.engine.get(which), b.engine.get(which))
+    assert a.delays == b.delays
+    a.close()
+    b.close()

@@ -148,3 +148,75 @@ def test_gamma_execution_time_model_matches_the_papers_figures():
     assert len(s1) == 500 and set(s1) == set(range(8)) and s1 == W.schedule_gamma(5, 8, 500)
     counts = np.bincount(W.schedule_gamma(5, 16, 4000, heterogeneous=True), minlength=16)
     assert counts.max() / max(1, counts.min()) > 2
+
+
+# ----------------------------------------------------------------------------- exact pins of the C generator
+def _round_f32(q):
+    """The fp32 value nearest to the exact rational q (ties to even), via exact comparisons."""
+    from fractions import Fraction
+    f = np.float32(float(q))
+    best = None
+    for c in (np.nextafter(f, np.float32(-np.inf)), f, np.nextafter(f, np.float32(np.inf))):
+        err = abs(Fraction(float(c)) - q)
+        even = (int(np.float32(c).view(np.uint32)) & 1) == 0
+        if best is None or err < best[0] or (err == best[0] and even):
+            best = (err, np.float32(c))
+    return best[1]
+
+
+def _exact_uniform(w):
+    from fractions import Fraction
+    return Fraction(2 * (w >> 41) + 1, 1 << 24)
+
+
+def _xi_f32(w):
+    from fractions import Fraction
+    fields = sum((w >> (16 * f)) & 0xFFFF for f in range(4)) - 131070
+    scale = np.float32(np.sqrt(3.0) / 65536.0)
+    return _round_f32(Fraction(fields) * Fraction(float(scale)))
+
+
+def test_generator_values_against_exact_arithmetic():
+    """Initial parameters, targets, curvature and gradients of the C generator at a handful of
+    elements, recomputed here from the Python statement of the hash and exact rational
+    arithmetic rounded once per operation: pins the C code to the written definition
+    independently of the device generator."""
+    from fractions import Fraction as F
+    wl = W.config("mini")
+    idx = np.array([0, 1, 999, 1000, 1036, 1037, 5135, 5136, 5137, 5652], dtype=np.int64)
+    t0, ts, a = wl.theta0(idx), wl.theta_star(idx), wl.curvature(idx)
+    sent = (t0 * np.float32(1.25)).astype(np.float32)
+    for k in (1, 9):
+        g = wl.grad(k, sent, idx)
+        for q, j in enumerate(int(x) for x in idx):
+            xi0 = _xi_f32(W.hash4(wl.seed, W.INIT, 0, j))
+            assert t0[q] == _round_f32(F(float(np.float32(0.05))) * F(float(xi0)))
+            xit = _xi_f32(W.hash4(wl.seed, W.TARGET, 0, j))
+            target = _round_f32(F(float(np.float32(0.1))) * F(float(xit)))
+            assert ts[q] == target
+            u = _exact_uniform(W.hash4(wl.seed, W.CURV, 0, j))
+            assert float(u) == float(np.float32(float(u)))          # the uniform is exact in fp32
+            curv = _round_f32(F(3, 2) * u + F(1, 2))
+            assert a[q] == curv
+            seg = int(np.searchsorted(wl.seg_off, j, side="right") - 1)
+            noise = _round_f32(F(float(wl.seg_sigma[seg])) * F(float(_xi_f32(W.hash4(wl.seed, W.NOISE, k, j)))))
+            diff = _round_f32(F(float(sent[q])) - F(float(target)))
+            want = _round_f32(F(float(curv)) * F(float(diff)) + F(float(noise)))       # one fused operation
+            assert g[q] == want, (k, j)
+
+
+def test_sparse_rows_follow_the_row_hash():
+    wl = W.Workload(name="emb", segments=[64 * 50, 500], n_workers=2, arrivals=4, schedule_kind="ticks",
+                    seed=11, quad=False, emb_rows=50, emb_row=64, row_active_frac=0.3)
+    g = wl.grad(3, np.zeros(wl.d, np.float32))
+    thresh = (1 << 64) * 300 // 1000
+    for r in range(50):
+        active = W.hash4(wl.seed, W.ROW, 3, r) < thresh
+        row = g[64 * r:64 * (r + 1)]
+        if active:
+            for c in (0, 63):
+                j = 64 * r + c
+                assert row[c] == np.float32(wl.seg_sigma[0]) * _xi_f32(W.hash4(wl.seed, W.NOISE, 3, j))
+        else:
+            assert not row.any()
+    assert (g[64 * 50:] != 0).mean() > 0.99

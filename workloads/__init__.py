@@ -3,8 +3,9 @@
 Input generation only: parameter-vector shapes (layer segments), arrival schedules of N
 simulated asynchronous workers, initial parameters and the stand-in worker gradient. None of
 the master's update arithmetic lives here. Both the CPU oracle's tests and the CUDA library's
-callers draw their inputs from this module; the per-element generators (wl_gen.h) are
-compiled once for the CPU (wl_cpu.c) and once for the device (wl_cuda.cu).
+callers draw their inputs from this module. The per-element generators exist twice, written
+separately from one definition: wl_cpu.c (plain C, feeds the oracle) and wl_gen.h + wl_cuda.cu
+(device); this module's own mix64/key/word in Python is a third statement used by the tests.
 
 The five workloads take the SHAPES of the models the paper trains (CIFAR ResNet-20, ImageNet
 ResNet-50, WRN-16-4, a Transformer language model); no dataset, model or weight is involved.
@@ -209,7 +210,7 @@ class _Spec(ctypes.Structure):
 
 
 def build_cpu(force=False):
-    srcs = [os.path.join(_HERE, "wl_cpu.c"), os.path.join(_HERE, "wl_gen.h")]
+    srcs = [os.path.join(_HERE, "wl_cpu.c")]
     if not force and os.path.exists(_CPU_LIB) and all(
             os.path.getmtime(_CPU_LIB) >= os.path.getmtime(s) for s in srcs):
         return _CPU_LIB

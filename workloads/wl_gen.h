@@ -1,8 +1,9 @@
 /* Seeded synthetic inputs for the parameter-server update: initial parameters, the
  * stand-in "worker" gradient and the per-segment noise scales. Input generation only:
- * nothing of the master's update rule lives here. The same inline functions are compiled
- * by gcc (CPU, wl_cpu.c) and by nvcc (device, wl_cuda.cu) so that the CPU oracle and the
- * CUDA library can be fed bit-identical inputs.
+ * nothing of the master's update rule lives here. This header is the DEVICE generator
+ * (compiled by nvcc into wl_cuda.cu); the CPU side that feeds the oracle is a separate program,
+ * wl_cpu.c, written from the same definitions and sharing no source with this file. A GPU test
+ * holds the two to bit-identical outputs.
  *
  * Every random quantity is a pure function of (seed, stream tag, a, b):
  *
