@@ -30,9 +30,11 @@ sys.path.insert(0, ROOT)
 METRIC = "ga_master_param_updates_per_sec"
 UNIT = "param-updates/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the last
-# ncu capture (profiles/), keyed by (variant, window); None once the kernel changed since.
-NCU_TRAFFIC_BYTES_PER_PARAM = {("GA", 16, "exact"): 212.6}   # profiles/ga_window_kernel_16M_k16_full.md
+# DRAM bytes per parameter per full window of the dominant kernel, from an ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum); the file also records a digest of the kernel
+# source at capture time, and the figure is dropped once the source has changed since.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ga_window_kernel_dram_traffic.json")
+KERNEL_SOURCE = os.path.join(ROOT, "paper_1909_10802_b200", "csrc", "ga_kernels.cuh")
 
 
 def parse_args():
@@ -47,10 +49,9 @@ def parse_args():
     ap.add_argument("--variant", default="GA", choices=["GA", "SA", "ASGD", "SA_GRAD", "DANA", "DANA_SA", "DANA_GA", "ADAM", "ADAM_SA", "ADAM_GA", "GA_LAYER"])
     ap.add_argument("--window", type=int, default=16)
     ap.add_argument("--math", default="exact", choices=["exact", "fast"])
-    ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--e2e-window", type=int, default=8)
-    ap.add_argument("--probe-hbm", action="store_true",
-                    help="print the bandwidth of plain torch kernels (copy, add, sum, fill) on this GPU and exit")
+    ap.add_argument("--e2e-steps", type=int, default=4, help="timed ga_push_batch_host calls")
+    ap.add_argument("--e2e-window", type=int, default=8, help="arrivals per fused window of the e2e leg")
+    ap.add_argument("--e2e-windows-per-step", type=int, default=2, help="windows handed over per call")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-params", type=int, default=4_000_000)
@@ -60,8 +61,8 @@ def parse_args():
 def bytes_per_param_window(variant, k):
     """Algorithmic bytes one parameter moves in a k-arrival window (fp32): theta, v (and m) in
     and out once; per arrival the gradient (and, for GA, the saved copy) in and the saved copy out."""
-    if variant == "GA_LAYER":                  # per arrival: norm pass 8 B, update pass 24 B; nothing fused in time
-        return 32 * k
+    if variant == "GA_LAYER":                  # one distance pass per call (8 B), then 28 B per arrival: theta, v, g and
+        return 8 + 28 * k                      # the next worker's copy in; theta, v and the sent copy out
     gap = variant in ("GA", "DANA_GA", "ADAM_GA")
     state = 24 if gap else 16                  # theta, v or sum_j v^j or Adam's m (, m behind C) in and out
     if variant.startswith("ADAM"):
@@ -70,6 +71,41 @@ def bytes_per_param_window(variant, k):
     if variant.startswith("DANA"):
         per_arrival += 8                                           # the worker's v^i in and out
     return state + per_arrival * k
+
+
+def measured_traffic(variant, window, math):
+    """(DRAM bytes per parameter of a full window from the last ncu capture, where it came from),
+    or (None, why not)."""
+    import hashlib
+    try:
+        with open(TRAFFIC_FILE) as f:
+            table = json.load(f)
+        entry = table["captures"][f"{variant}/{window}/{math}"]
+    except Exception:
+        return None, "no ncu capture on record for this variant, window and math mode"
+    with open(KERNEL_SOURCE, "rb") as f:
+        digest = hashlib.sha256(f.read()).hexdigest()
+    if digest != entry.get("kernel_source_sha256"):
+        return None, "kernel source changed since the ncu capture"
+    return float(entry["dram_bytes_per_param"]), entry.get("source", os.path.relpath(TRAFFIC_FILE, ROOT))
+
+
+def host_cpu():
+    """(usable cores, CPU model string) of this machine."""
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except AttributeError:
+        cores = os.cpu_count() or 1
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return cores, model
 
 
 def hbm_peak():
@@ -153,18 +189,21 @@ def bench_windows(wl, window, count):
 
 
 # ------------------------------------------------------------------------------ CPU oracle legs
-def time_oracle(wl, variant, n_params, windows_list, seed_offset=0):
+def time_oracle(wl, variant, n_params, windows_list, all_cores=False):
     """The oracle, as it stands, on a contiguous slice of the workload's parameter vector.
     Only push+pull are timed (gradients are generated beforehand), like the GPU's timed region.
-    Returns (param_updates, seconds)."""
+    all_cores: the same source built with OpenMP (loops over parameters split across threads).
+    Returns (param_updates, seconds, description)."""
     import numpy as np
     import oracle
+    lib = oracle.lib_openmp() if all_cores else None
+    threads = host_cpu()[0] if all_cores else 1
     n_params = min(n_params, wl.d)
     j0 = max(0, wl.spec.emb_elems - n_params // 2) if wl.spec.emb_elems else 0   # straddle embedding/dense
     j0 = min(j0, wl.d - n_params)
     idx = np.arange(j0, j0 + n_params, dtype=np.int64)
     o = oracle.Oracle(n_params, wl.n_workers, wl.lr, wl.momentum, wl.c_beta,
-                      oracle.VARIANTS[variant], precision=32)
+                      oracle.VARIANTS[variant], precision=32, _lib=lib)
     o.set_params(wl.theta0(idx))
     k, updates, seconds = 0, 0, 0.0
     for win in windows_list:
@@ -174,8 +213,28 @@ def time_oracle(wl, variant, n_params, windows_list, seed_offset=0):
         seconds += time.perf_counter() - t0
         k += len(win)
         updates += len(win) * n_params
-    return updates, seconds, f"oracle (fp32, 1 thread) on parameters [{j0}, {j0 + n_params}) of {wl.name}, " \
-                             f"{k} arrivals push+pull"
+    return updates, seconds, f"oracle (fp32, {threads} thread{'s' if threads > 1 else ''}) on parameters " \
+                             f"[{j0}, {j0 + n_params}) of {wl.name}, {k} arrivals push+pull"
+
+
+def cpu_baseline_legs(wl, variant, window, sample_params):
+    """The cpu_baseline object: the oracle on one thread and, from the same source built with
+    OpenMP, on all host cores, each on a bounded slice of the workload."""
+    cores, model = host_cpu()
+    cw = bench_windows(wl, window, 3)
+    time_oracle(wl, variant, min(sample_params, wl.d) // 8, cw[:1])
+    updates, seconds, sample = time_oracle(wl, variant, sample_params, cw)
+    out = {"value": updates / seconds, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+           "host_cores": cores, "cpu_model": model}
+    try:
+        os.environ.setdefault("OMP_NUM_THREADS", str(cores))
+        time_oracle(wl, variant, min(sample_params, wl.d), cw[:1], all_cores=True)
+        u2, s2, sample2 = time_oracle(wl, variant, min(4 * sample_params, wl.d), cw, all_cores=True)
+        out["all_cores"] = {"value": u2 / s2, "unit": UNIT, "cores": cores, "kind": "oracle built with OpenMP",
+                            "sample": sample2}
+    except Exception as exc:                      # no OpenMP runtime on this machine
+        out["all_cores"] = {"unavailable": str(exc)[:200]}
+    return out
 
 
 def run_reference(args):
@@ -196,7 +255,8 @@ def run_reference(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{wl.name}: {wl.d} fp32 params, {wl.n_workers} workers, {args.variant}, "
                                f"window {args.window}", "note": "each step = one window on a bounded slice"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": host_cpu()[0], "cpu_model": host_cpu()[1]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -276,13 +336,13 @@ def run_ours(args):
     achieved = alg_bytes / (sum(ms) * 1e-3) / 1e9
     peak, peak_src = hbm_peak()
     full = [(m, n) for m, (_, _, n) in zip(ms, events) if n == args.window]
-    traffic_pp = NCU_TRAFFIC_BYTES_PER_PARAM.get((args.variant, args.window, args.math))
+    traffic_pp, traffic_src = measured_traffic(args.variant, args.window, args.math)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 # measured DRAM bytes of a full window, scaled to the average launch of this run
                 # (windows cut short by a repeated worker move proportionally fewer bytes)
                 "traffic": (traffic_pp * wl.d * (alg_bytes / max(1, launches)) /
                             (bytes_per_param_window(args.variant, args.window) * wl.d)) if traffic_pp else None,
-                "peak_source": peak_src,
+                "traffic_source": traffic_src, "peak_source": peak_src,
                 "kernel": "ga_window_kernel", "algorithmic_bytes_per_launch": alg_bytes / max(1, launches),
                 "avg_launch_ms": sum(ms) / max(1, launches),
                 "frac_of_nominal_8TBs": achieved / 8000.0,
@@ -296,10 +356,7 @@ def run_ours(args):
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cw = bench_windows(base, args.window, 3)
-        time_oracle(base, args.variant, min(args.cpu_sample_params, base.d) // 8, cw[:1])
-        updates, seconds, sample = time_oracle(base, args.variant, args.cpu_sample_params, cw)
-        cpu_baseline = {"value": updates / seconds, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample}
+        cpu_baseline = cpu_baseline_legs(base, args.variant, args.window, args.cpu_sample_params)
 
     if rank == 0:
         line = {
@@ -321,28 +378,63 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def pcie_rates(host_in, dev_in, dev_out, host_out, repeats=3):
+    """What plain copies reach on this machine: one pinned host->device copy and one device->pinned
+    host copy of whole vectors running at the same time on two streams (the traffic pattern of the
+    end-to-end path). Returns (host->device GB/s, device->host GB/s), best of `repeats`."""
+    import torch
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    best = [0.0, 0.0]
+    nbytes = host_in.numel() * 4
+    for _ in range(repeats + 1):
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        with torch.cuda.stream(s_in):
+            ev[0].record(s_in)
+            dev_in.copy_(host_in, non_blocking=True)
+            ev[1].record(s_in)
+        with torch.cuda.stream(s_out):
+            ev[2].record(s_out)
+            host_out.copy_(dev_out, non_blocking=True)
+            ev[3].record(s_out)
+        torch.cuda.synchronize()
+        best[0] = max(best[0], nbytes / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9)
+        best[1] = max(best[1], nbytes / (ev[2].elapsed_time(ev[3]) * 1e-3) / 1e9)
+    return best[0], best[1]
+
+
 def run_e2e(args, run, wl, base, world, dist, barrier):
     """Same metric through ga_push_batch_host: gradients start in pinned host memory and the
-    parameters sent back to each worker end in pinned host memory, copies inside the timed region."""
+    parameters sent back to each worker end in pinned host memory, copies inside the timed region.
+    One step = one call that hands over several fused windows."""
     import torch
     k = min(args.e2e_window, args.window)
-    wins = bench_windows(base, k, args.e2e_steps + 1)      # the replicated schedule
+    wps = args.e2e_windows_per_step
+    if world > 1:            # every rank pins its own buffers: keep the node's pinned memory small
+        k, wps = min(k, 2), 2
+    wins = bench_windows(base, k, (args.e2e_steps + 1) * wps)      # the replicated schedule
+    steps = [[i for w in wins[q * wps:(q + 1) * wps] for i in w] for q in range(args.e2e_steps + 1)]
     grads = [torch.empty(wl.d, dtype=torch.float32).pin_memory() for _ in range(k)]
     outs = [torch.empty(wl.d, dtype=torch.float32).pin_memory() for _ in range(k)]
     for j, g in enumerate(grads):                     # synthetic gradients, generated on the device
         run.dev.grad_ptr(run.k + 1 + j, run.engine.saved_ptr(wins[0][j % len(wins[0])]), run.grads[0].data_ptr())
         g.copy_(run.grads[0])
     torch.cuda.synchronize()
-    run.engine.push_batch_host(wins[0], grads[:len(wins[0])], outs[:len(wins[0])])     # warm-up
+
+    def call(sched):
+        n = len(sched)
+        run.engine.push_batch_host(sched, [grads[q % k] for q in range(n)], [outs[q % k] for q in range(n)])
+        return n
+
+    call(steps[0])                                    # warm-up (allocates the staging buffers)
     barrier()
     stream = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     arrivals = 0
     t0 = time.perf_counter()
     e0.record(stream)
-    for win in wins[1:]:
-        run.engine.push_batch_host(win, grads[:len(win)], outs[:len(win)])
-        arrivals += len(win)
+    for sched in steps[1:]:
+        arrivals += call(sched)
     e1.record(stream)
     barrier()
     seconds = max(e0.elapsed_time(e1) * 1e-3, time.perf_counter() - t0 if world == 1 else 0.0)
@@ -351,42 +443,20 @@ def run_e2e(args, run, wl, base, world, dist, barrier):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         seconds = float(t.item())
     per_step = arrivals / max(1, args.e2e_steps)
+    bytes_each_way = arrivals * wl.d * 4
+    h2d, d2h = pcie_rates(grads[0], run.grads[0], run.grads[-1], outs[0])   # outside the timed region
+    bound = max(bytes_each_way / (h2d * 1e9), bytes_each_way / (d2h * 1e9))
     return {"value": arrivals * wl.d * world / seconds, "unit": UNIT,
             "h2d_bytes_per_step": int(per_step * wl.d * 4), "d2h_bytes_per_step": int(per_step * wl.d * 4),
-            "steps": args.e2e_steps, "window": k,
+            "steps": args.e2e_steps, "window": k, "windows_per_step": wps,
+            "pcie_h2d_gbs": h2d, "pcie_d2h_gbs": d2h, "pcie_frac": bound / seconds,
+            "pcie_note": "plain pinned copies of one vector each way, concurrently on two streams, best of 3; "
+                         "pcie_frac = time those rates need for this leg's bytes / measured time",
             "note": "ga_push_batch_host: pinned host gradients in, sent parameters out, chunked overlap"}
-
-
-def probe_hbm():
-    """Context for the roofline denominator: what library kernels with simple read/write mixes
-    reach on this GPU (4 GiB fp32 vectors, best of 10, CUDA events)."""
-    import torch
-    n = 1 << 30
-    a, b = torch.randn(n, device="cuda"), torch.randn(n, device="cuda")
-    c = torch.empty_like(a)
-    out = {}
-    for name, fn, nbytes in (("copy_1r1w", lambda: c.copy_(a), 8 * n), ("add_2r1w", lambda: torch.add(a, b, out=c), 12 * n),
-                             ("sum_read_only", lambda: a.sum(), 4 * n), ("fill_write_only", lambda: c.fill_(1.0), 4 * n)):
-        for _ in range(3):
-            fn()
-        torch.cuda.synchronize()
-        best = float("inf")
-        for _ in range(10):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            fn()
-            e1.record()
-            torch.cuda.synchronize()
-            best = min(best, e0.elapsed_time(e1))
-        out[name] = round(nbytes / best / 1e6, 1)
-    print(json.dumps({"probe": "hbm_gbs_of_torch_kernels", **out}), flush=True)
 
 
 def main():
     args = parse_args()
-    if args.probe_hbm:
-        probe_hbm()
-        return
     if args.impl == "reference":
         run_reference(args)
     else:

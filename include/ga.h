@@ -229,6 +229,24 @@ int64_t ga_worker_iter(ga_engine* e, int worker);
 size_t ga_export_state(ga_engine* e, void* buf_host, size_t cap);
 int ga_import_state(ga_engine* e, const void* buf_host, size_t len);
 
+/* Self-test of the kernels' exact arithmetic on the current device. In exact mode (GA_OPT_MATH = 0)
+ * the Gap-Aware kernels evaluate the square root in C (Algorithm "C Coefficient Calculation"), the
+ * division and the reciprocal of the Gap (Algorithm "Gap-Aware: master") and Adam's root and division
+ * (Algorithm "Adam-Gap-Aware: master") by short sequences -- hardware seed, one Newton step, one
+ * residual correction -- wherever the operands lie in ranges for which those sequences return
+ * the IEEE round-to-nearest result, and by the general IEEE routines elsewhere. That claim rests on
+ * the GPU's approximate reciprocal and reciprocal square root as well as on arithmetic, so this call
+ * repeats the comparison with the IEEE routines on the device at hand:
+ *   level 0 (well under a second): the reciprocal for every value in [2^-100, 2^100]; the square
+ *     root for every value in [2^-100, FLT_MAX] and at 0; the division for 2 x 10^9 random significand
+ *     pairs spread over every exponent pair of the windows the kernels use, for constant numerators
+ *     over every divisor in [1, 2^100], and for tiny and subnormal distances;
+ *   level 1 (about a minute): additionally the division for all 2^46 pairs of significands.
+ * Returns the number of operands on which a short form differs from IEEE (0 on a B200), or a
+ * negative GA_ERR_* code. Allocates 8 bytes of device memory for the duration of the call and
+ * synchronises cuda_stream. */
+int64_t ga_selftest_exact_forms(int level, void* cuda_stream);
+
 /* Gap statistics without any allocation. (The paper has no counterpart of this call; it exists
  * for deployment reasons only.) Computes the sum and the maximum over all parameters of the
  * parameter-wise Gap |theta - saved| / C + 1, with C = lr_max * (sqrt(m / (1 - c_beta^n_refreshes))

@@ -56,6 +56,7 @@ _SIGNATURES = {
     "ga_import_state": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_size_t]),
     "ga_gap_stats_noalloc": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_size_t, _c.c_float, _c.c_float,
                                         _c.c_int64, _c.c_void_p, _c.c_void_p]),
+    "ga_selftest_exact_forms": (_c.c_int64, [_c.c_int, _c.c_void_p]),
     "ga_last_error": (_c.c_char_p, []),
 }
 
@@ -114,6 +115,14 @@ def gap_stats_noalloc(theta, saved, m, lr_max, c_beta, n_refreshes, out, stream=
     _check(lib().ga_gap_stats_noalloc(theta.data_ptr(), saved.data_ptr(), m.data_ptr(), n, lr_max, c_beta,
                                       n_refreshes, out.data_ptr(), raw))
     return out
+
+
+def selftest_exact_forms(level=0, stream=None):
+    """ga_selftest_exact_forms: operands on which the kernels' short exact forms differ from the
+    IEEE routines on the current device (0 = they agree everywhere they are used)."""
+    import torch
+    raw = (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+    return _check(lib().ga_selftest_exact_forms(level, raw))
 
 
 class Engine:

@@ -14,6 +14,7 @@
 
 #include "ga_kernels.cuh"
 #include "ga_layer_kernels.cuh"
+#include "ga_selftest.cuh"
 
 namespace {
 
@@ -48,9 +49,14 @@ struct ga_engine {
     std::vector<int64_t> layer_off;
     ga::Tile* tiles = nullptr;
     int* tile_begin = nullptr;     // n_layers + 1
-    double* tile_partial = nullptr;
+    double* tile_partial = nullptr;   // 2 x n_tiles: sums of v^2, then sums of squared distances
+    unsigned int* layer_ticket = nullptr;
     float *m_layer = nullptr, *layer_gap = nullptr, *layer_inv_gap = nullptr;
     int n_tiles = 0;
+    ga::LayerTables layer_tables() const {
+        return ga::LayerTables{tiles, tile_begin, tile_partial, tile_partial + n_tiles, layer_ticket, m_layer,
+                               layer_gap, layer_inv_gap};
+    }
     bool is_layer() const { return variant == GA_GA_LAYER; }
     int n_layers() const { return (int)layer_off.size() - 1; }
     float* sec = nullptr;         // Adam: second moment (vel holds the first moment, gamma is beta_1)
@@ -98,6 +104,8 @@ struct ga_engine {
         h.adam_eps = adam_eps;
         h.wd = weight_decay;
         h.nesterov = nesterov;
+        h.short_forms = ga::short_forms_ok(lr_max, eps, is_adam() ? adam_eps : 1e-8f,
+                                           is_adam() ? h.one_minus_gamma : 1.0f) ? 1 : 0;
         return h;
     }
     // (float)(1 / (1 - base^k)), base^k = pow(base, k) in double. Consecutive k reuse the previous
@@ -185,7 +193,6 @@ int grid_1d(long long n, int threads, int cap) {
 }
 
 // ----------------------------------------------------------------------------- launch
-int launch_layer_arrival(ga_engine* e, const float* grad, float* saved_row, bool write_saved, float inv_bias);
 
 // stats_mode (STATS instantiations): 1 = the arrivals' pairs overwrite their log slots, 2 = they are
 // merged into them (a later chunk of the same arrivals on the host-buffer path)
@@ -196,8 +203,7 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
     long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
     // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner.
-    // Exact Adam-GA is bound by its arithmetic, not by loads in flight: it keeps the register path.
-    constexpr int ST = (FAMILY == ga::ADAM && PENALTY == ga::PEN_GAP && EXACT) ? 0 : GA_WINDOW_STAGES;
+    constexpr int ST = GA_WINDOW_STAGES;
 #define GA_LAUNCH(BATCH, STAGES_, WD_)                                                                          \
     ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, BATCH, STAGES_, WD_>                            \
         <<<(unsigned)blocks, ga::kThreads, 0, st>>>(e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, \
@@ -238,13 +244,7 @@ void launch_family(ga_engine* e, const ga::Window& w, long long vb, long long ve
 int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st,
                   bool first_range = true, bool last_range = true) {
     if (vec_end <= vec_begin || w.K <= 0) return GA_OK;
-    if (e->is_layer()) {   // a layer's norm needs the whole vector between arrivals: no fusion in time
-        if (vec_begin != 0 || vec_end != e->stride / 4)
-            return fail(GA_ERR_STATE, "the layer-wise Gap cannot run on a sub-range of the vector");
-        for (int j = 0; j < w.K; ++j)
-            if (int rc = launch_layer_arrival(e, w.grad[j], w.saved[j], w.write_saved != 0, w.inv_bias[j])) return rc;
-        return GA_OK;
-    }
+    if (e->is_layer()) return fail(GA_ERR_STATE, "the layer-wise Gap takes whole arrivals: see launch_layer_arrivals");
     const int stats = (e->stats && e->is_gap()) ? (first_range ? 1 : 2) : 0;
     if (e->is_dana()) launch_family<ga::DANA>(e, w, vec_begin, vec_end, st, stats);
     else if (e->is_adam()) launch_family<ga::ADAM>(e, w, vec_begin, vec_end, st, stats);
@@ -255,9 +255,9 @@ int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long l
 }
 
 void free_layers(ga_engine* e) {
-    cudaFree(e->tiles); cudaFree(e->tile_begin); cudaFree(e->tile_partial);
+    cudaFree(e->tiles); cudaFree(e->tile_begin); cudaFree(e->tile_partial); cudaFree(e->layer_ticket);
     cudaFree(e->m_layer); cudaFree(e->layer_gap); cudaFree(e->layer_inv_gap);
-    e->tiles = nullptr; e->tile_begin = nullptr; e->tile_partial = nullptr;
+    e->tiles = nullptr; e->tile_begin = nullptr; e->tile_partial = nullptr; e->layer_ticket = nullptr;
     e->m_layer = e->layer_gap = e->layer_inv_gap = nullptr;
     e->n_tiles = 0;
 }
@@ -281,7 +281,8 @@ int build_layers(ga_engine* e, const int64_t* offsets, int n) {
     const size_t nt = tiles.size();
     bool ok = cudaMalloc(&e->tiles, sizeof(ga::Tile) * nt) == cudaSuccess &&
               cudaMalloc(&e->tile_begin, sizeof(int) * (n + 1)) == cudaSuccess &&
-              cudaMalloc(&e->tile_partial, sizeof(double) * nt) == cudaSuccess &&
+              cudaMalloc(&e->tile_partial, sizeof(double) * 2 * nt) == cudaSuccess &&
+              cudaMalloc(&e->layer_ticket, sizeof(unsigned int) * n) == cudaSuccess &&
               cudaMalloc(&e->m_layer, sizeof(float) * n) == cudaSuccess &&
               cudaMalloc(&e->layer_gap, sizeof(float) * n) == cudaSuccess &&
               cudaMalloc(&e->layer_inv_gap, sizeof(float) * n) == cudaSuccess;
@@ -294,21 +295,30 @@ int build_layers(ga_engine* e, const int64_t* offsets, int n) {
     GA_CUDA(e, cudaMemcpy(e->tile_begin, begin.data(), sizeof(int) * (n + 1), cudaMemcpyHostToDevice));
     GA_CUDA(e, cudaMemset(e->m_layer, 0, sizeof(float) * n));
     GA_CUDA(e, cudaMemset(e->layer_gap, 0, sizeof(float) * n));
+    GA_CUDA(e, cudaMemset(e->layer_ticket, 0, sizeof(unsigned int) * n));
     e->layer_off.assign(offsets, offsets + n + 1);
     e->n_tiles = (int)nt;
     return GA_OK;
 }
 
-// One arrival with the layer-wise Gap: two passes over the vector and two per-layer steps.
-int launch_layer_arrival(ga_engine* e, const float* grad, float* saved_row, bool write_saved, float inv_bias) {
+// Arrivals w.K of a window with the layer-wise Gap, one launch each. The Gap of the window's
+// first arrival is in place already when `primed` (the previous launch computed it); otherwise a
+// distance pass computes it first. `next_row` / `next_inv_bias` describe the arrival that follows
+// the window inside the same call (nullptr: none is known), so that the last launch of this window
+// can prepare its Gap as well.
+int launch_layer_arrivals(ga_engine* e, const ga::Window& w, bool primed, const float* next_row, float next_inv_bias) {
     const ga::Hyper h = e->hyper();
-    const int P = e->n_layers();
-    ga::ga_layer_dist_kernel<<<e->n_tiles, ga::kLayerThreads, 0, e->stream>>>(e->theta, saved_row, e->tiles, e->tile_partial);
-    ga::ga_layer_gap_kernel<<<P, ga::kLayerThreads, 0, e->stream>>>(e->tile_partial, e->tile_begin, e->m_layer, inv_bias, h,
-                                                                    e->layer_gap, e->layer_inv_gap);
-    ga::ga_layer_update_kernel<<<e->n_tiles, ga::kLayerThreads, 0, e->stream>>>(
-        e->theta, e->vel, grad, saved_row, write_saved ? 1 : 0, e->tiles, e->layer_inv_gap, e->lr, h, e->tile_partial);
-    ga::ga_layer_refresh_kernel<<<P, ga::kLayerThreads, 0, e->stream>>>(e->tile_partial, e->tile_begin, e->m_layer, h);
+    const ga::LayerTables T = e->layer_tables();
+    if (!primed)
+        ga::ga_layer_dist_kernel<<<e->n_tiles, ga::kLayerThreads, 0, e->stream>>>(e->theta, w.saved[0], T, w.inv_bias[0], h);
+    for (int j = 0; j < w.K; ++j) {
+        const float* nxt = j + 1 < w.K ? w.saved[j + 1] : next_row;
+        const float nxt_ib = j + 1 < w.K ? w.inv_bias[j + 1] : next_inv_bias;
+        // the same worker again right away: its saved copy is the theta this launch writes, distance 0
+        const int mode = !nxt ? 0 : (nxt == w.saved[j] && w.write_saved) ? 2 : 1;
+        ga::ga_layer_update_kernel<<<e->n_tiles, ga::kLayerThreads, 0, e->stream>>>(
+            e->theta, e->vel, w.grad[j], w.saved[j], w.write_saved, nxt, mode, T, e->lr, h, nxt_ib);
+    }
     GA_CUDA(e, cudaGetLastError());
     return GA_OK;
 }
@@ -594,6 +604,10 @@ int64_t ga_push(ga_engine* e, int worker, const float* grad_dev) {
     int64_t tau = 0;
     e->stats_total = 0;
     fill_window(e, w, &worker, &grad_dev, 1, /*with_pull=*/false, &tau);
+    if (e->is_layer()) {
+        if (int rc = launch_layer_arrivals(e, w, false, nullptr, 0.f)) return rc;
+        return tau;
+    }
     if (int rc = launch_window(e, w, 0, e->stride / 4, e->stream)) return rc;
     return tau;
 }
@@ -605,6 +619,29 @@ int ga_push_batch(ga_engine* e, const int* schedule_host, const float* const* gr
     DeviceGuard guard(e->device);
     int launches = 0;
     if (K > 0) e->stats_total = 0;
+    if (e->is_layer()) {
+        // Arrivals are not fused in time (a layer's norm needs the whole vector between them), but
+        // each launch also measures the next arrival's distance: one launch per arrival after a
+        // first distance pass. The table is filled 16 arrivals at a time; a worker may repeat freely.
+        ga::Window cur, nxt;
+        int n_cur = K < ga::kMaxWindow ? K : ga::kMaxWindow;
+        if (K > 0) fill_window(e, cur, schedule_host, grads_host, n_cur, true, delays_out_host);
+        for (int pos = 0; pos < K;) {
+            const int after = pos + n_cur;
+            const int n_nxt = K - after < ga::kMaxWindow ? K - after : ga::kMaxWindow;
+            if (n_nxt > 0)
+                fill_window(e, nxt, schedule_host + after, grads_host + after, n_nxt, true,
+                            delays_out_host ? delays_out_host + after : nullptr);
+            if (int rc = launch_layer_arrivals(e, cur, pos > 0, n_nxt > 0 ? nxt.saved[0] : nullptr,
+                                               n_nxt > 0 ? nxt.inv_bias[0] : 0.f))
+                return rc;
+            launches += n_cur + (pos == 0 ? 1 : 0);
+            pos = after;
+            cur = nxt;
+            n_cur = n_nxt;
+        }
+        return launches;
+    }
     for (int pos = 0; pos < K;) {
         const int n = next_window(schedule_host, pos, K, e->window);
         ga::Window w;
@@ -937,6 +974,34 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len) {
 }
 
 }  // extern "C"
+
+// ============================================================ self-test of the short exact forms
+extern "C" int64_t ga_selftest_exact_forms(int level, void* cuda_stream) {
+    if (level < 0 || level > 1) return fail(GA_ERR_ARG, "level must be 0 or 1");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    unsigned long long* bad = nullptr;
+    if (cudaMalloc(&bad, sizeof *bad) != cudaSuccess) { cudaGetLastError(); return fail(GA_ERR_OOM, "cannot allocate a counter"); }
+    auto done = [&](int64_t rc) { cudaFree(bad); return rc; };
+    if (cudaMemsetAsync(bad, 0, sizeof *bad, st) != cudaSuccess) return done(fail(GA_ERR_CUDA, "cudaMemsetAsync failed"));
+    namespace t = ga::selftest;
+    const int grid = 148 * 16, block = 256;
+    t::rcp_range<<<grid, block, 0, st>>>(0x3f800000u, 0x71800001u, bad);                 // every b in [1, 2^100]
+    t::rcp_range<<<grid, block, 0, st>>>(0x0d800000u, 0x3f800000u, bad);                 // every b in [2^-100, 1)
+    t::sqrt_range<<<grid, block, 0, st>>>(0x0d800000u, 0x7f800000u, 1e-8f, bad);          // every x in [2^-100, FLT_MAX]
+    t::div_window<<<grid, block, 0, st>>>(-100, 100, -100, 100, -124, 126, 1u << 14, 1, bad);   // 6.6e8 pairs
+    t::div_window<<<grid, block, 0, st>>>(-101, 127, -76, 105, -25, 100, 1u << 14, 2, bad);     // dist / C
+    t::div_window<<<grid, block, 0, st>>>(-60, 60, -27, 65, -124, 87, 1u << 15, 3, bad);        // Adam's step
+    for (float c : {0.1f, 0.01f, 1.0f, 0.001f, 0.5f}) t::div_const<<<grid, block, 0, st>>>(c, bad);
+    t::gap_small_dist<<<grid, block, 0, st>>>(1u << 20, 4, bad);
+    if (level >= 1)
+        for (uint32_t slice = 0; slice < 64; ++slice) t::div_all_significands<<<1024, 128, 0, st>>>(slice << 17, bad);
+    unsigned long long host = 0;
+    cudaError_t err = cudaGetLastError();
+    if (err == cudaSuccess) err = cudaMemcpyAsync(&host, bad, sizeof host, cudaMemcpyDeviceToHost, st);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(st);
+    if (err != cudaSuccess) return done(fail(GA_ERR_CUDA, "ga_selftest_exact_forms: %s", cudaGetErrorString(err)));
+    return done((int64_t)host);
+}
 
 // ============================================================ allocation-free Gap statistics
 // Everything this entry point needs lives in this file: the scratch array is part of the

@@ -359,3 +359,65 @@ def test_import_state_refuses_inconsistent_headers(P):
     assert a.delays == b.delays
     a.close()
     b.close()
+
+
+# ----------------------------------------------------------------------------- exact arithmetic
+def test_short_exact_forms_agree_with_ieee_on_this_device(P):
+    """Exact mode evaluates roots, divisions and reciprocals by short sequences wherever their
+    operands lie in proven ranges. The library's self-test compares them with the IEEE routines on
+    this GPU: every reciprocal operand in [2^-100, 2^100], every radicand in [2^-100, FLT_MAX],
+    2 x 10^9 random divisions over all exponent pairs of the windows in use, constant numerators over
+    every divisor in [1, 2^100]. Not one operand may differ."""
+    assert P.selftest_exact_forms(0) == 0
+    assert P.lib().ga_selftest_exact_forms(7, None) == P.GA_ERR_ARG
+
+
+@pytest.mark.parametrize("variant", ["GA", "DANA_GA", "ADAM_GA", "ADAM"])
+def test_short_forms_and_ieee_fallback_give_the_same_bits(P, variant):
+    """The same three arrivals with hyper-parameters inside the proven ranges (short forms on) and
+    from a checkpoint whose eta_max lies outside them (every element takes the IEEE routines): both
+    must equal the oracle bit for bit, on values spanning tiny, ordinary and huge magnitudes."""
+    import torch
+    d, n = 40_000, 3
+    rng = np.random.default_rng(5)
+    var = oracle.VARIANTS[variant]
+
+    def spread(nonneg=False):
+        x = (10.0 ** rng.uniform(-30, 20, size=d)) * (1 if nonneg else rng.choice([-1.0, 1.0], size=d))
+        x = x.astype(np.float32)
+        x[rng.integers(0, 10, size=d) == 0] = 0.0
+        return x
+
+    for lr_max in (0.1, 1e-20):                    # 1e-20 < 2^-49: outside the short forms' range
+        o = oracle.Oracle(d, n, lr_max, 0.9, 0.999, var)
+        eng = P.Engine(d, n, lr_max, 0.9, 0.999, var)
+        theta, v, m = spread(), spread(), spread(nonneg=True)
+        saved = np.stack([spread() for _ in range(n)])
+        saved[1, ::2] = theta[::2]
+        iters = np.array([1, 0, 3], dtype=np.int64)
+        extra = {}
+        if variant == "DANA_GA":
+            extra = dict(v_workers=np.stack([spread() for _ in range(n)]))
+        if variant.startswith("ADAM"):
+            extra = dict(v_workers=spread(nonneg=True))
+        o.set_state(theta, v, m, saved, iters, 4, 4, **extra)
+        st = P.unpack_state(eng.export_state())
+        st.update(theta=theta, v=v, m=m, saved=saved, iter=iters, k_done=4, k_c=4)
+        if variant == "DANA_GA":
+            st["v_workers"] = extra["v_workers"]
+        if variant.startswith("ADAM"):
+            st["v2"] = extra["v_workers"]
+        eng.import_state(P.pack_state(st))
+        grads = [spread() for _ in range(3)]
+        sched = [1, 0, 2]
+        assert eng.push_batch(sched, [torch.from_numpy(g).cuda() for g in grads]) == o.push_batch(sched, grads)
+        pairs = [(P.GA_THETA, o.get(o.THETA)), (P.GA_V, o.get(o.V))]
+        if variant != "ADAM":
+            pairs.append((P.GA_M, o.get(o.M)))
+        if variant.startswith("ADAM"):
+            pairs.append((P.GA_V2, o.second_moment()))
+        for which, ref in pairs:
+            got = _np(eng.get(which))
+            bad = ~((got == ref.astype(np.float32)) | (np.isnan(got) & np.isnan(ref)))
+            assert not bad.any(), (variant, lr_max, which, int(bad.sum()), got[bad][:4], ref[bad][:4])
+        eng.close()
