@@ -352,6 +352,13 @@ def test_import_state_refuses_inconsistent_headers(P):
         doctored = blob[:hs] + iters.tobytes() + blob[hs + 8 * wl.n_workers:]
         assert a.engine._l.ga_import_state(a.engine._h, doctored, len(doctored)) == P.GA_ERR_ARG
         assert "iter" in P.last_error()
+    # a second moment is a running average of squares: a negative entry is refused
+    st = P.unpack_state(blob)
+    st["m"] = st["m"].copy()
+    st["m"][17] = -1e-6
+    doctored = P.pack_state(st)
+    assert a.engine._l.ga_import_state(a.engine._h, doctored, len(doctored)) == P.GA_ERR_ARG
+    assert "second moment" in P.last_error()
     a.run()
     b.run()
     for which in (P.GA_THETA, P.GA_V, P.GA_M):
