@@ -51,11 +51,13 @@ struct ga_engine {
     int* tile_begin = nullptr;     // n_layers + 1
     double* tile_partial = nullptr;   // 2 x n_tiles: sums of v^2, then sums of squared distances
     unsigned int* layer_ticket = nullptr;
+    unsigned int* layer_epoch = nullptr;   // per layer: Gaps made ready so far; layer_epoch_host mirrors their common value
+    unsigned int layer_epoch_host = 0;
     float *m_layer = nullptr, *layer_gap = nullptr, *layer_inv_gap = nullptr;
     int n_tiles = 0;
     ga::LayerTables layer_tables() const {
-        return ga::LayerTables{tiles, tile_begin, tile_partial, tile_partial + n_tiles, layer_ticket, m_layer,
-                               layer_gap, layer_inv_gap};
+        return ga::LayerTables{tiles, tile_begin, tile_partial, tile_partial + n_tiles, layer_ticket, layer_epoch,
+                               m_layer, layer_gap, layer_inv_gap};
     }
     bool is_layer() const { return variant == GA_GA_LAYER; }
     int n_layers() const { return (int)layer_off.size() - 1; }
@@ -174,14 +176,16 @@ int check_dev_ptr(const void* p, const char* name) {
     return GA_OK;
 }
 
-// Every synchronising call ends here: wait for the engine's stream, then see whether a
-// bulk-copy wait of a pull kernel ran out (the kernel raises a flag in mapped host memory). Such
-// a pull left its saved copy incomplete, so the failure is sticky like a CUDA error.
+// Every synchronising call ends here: wait for the engine's stream, then see whether a bounded
+// wait inside a kernel ran out (a bulk copy of the pull kernel, or a layer's Gap in the layer-wise
+// kernel): the kernel then raised a flag in mapped host memory and left its work incomplete, so
+// the failure is sticky like a CUDA error.
 int sync_and_check(ga_engine* e) {
     GA_CUDA(e, cudaStreamSynchronize(e->stream));
-    if (*(volatile int*)e->pull_err) {
+    if (const int flag = *(volatile int*)e->pull_err) {
         e->cuda_failed = true;
-        return fail(GA_ERR_CUDA, "a bulk copy of ga_pull did not complete within its wait limit");
+        return fail(GA_ERR_CUDA, flag == 2 ? "a block of the layer-wise kernel gave up waiting for a layer's Gap"
+                                           : "a bulk copy of ga_pull did not complete within its wait limit");
     }
     return GA_OK;
 }
@@ -256,6 +260,8 @@ int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long l
 
 void free_layers(ga_engine* e) {
     cudaFree(e->tiles); cudaFree(e->tile_begin); cudaFree(e->tile_partial); cudaFree(e->layer_ticket);
+    cudaFree(e->layer_epoch);
+    e->layer_epoch = nullptr;
     cudaFree(e->m_layer); cudaFree(e->layer_gap); cudaFree(e->layer_inv_gap);
     e->tiles = nullptr; e->tile_begin = nullptr; e->tile_partial = nullptr; e->layer_ticket = nullptr;
     e->m_layer = e->layer_gap = e->layer_inv_gap = nullptr;
@@ -283,6 +289,7 @@ int build_layers(ga_engine* e, const int64_t* offsets, int n) {
               cudaMalloc(&e->tile_begin, sizeof(int) * (n + 1)) == cudaSuccess &&
               cudaMalloc(&e->tile_partial, sizeof(double) * 2 * nt) == cudaSuccess &&
               cudaMalloc(&e->layer_ticket, sizeof(unsigned int) * n) == cudaSuccess &&
+              cudaMalloc(&e->layer_epoch, sizeof(unsigned int) * n) == cudaSuccess &&
               cudaMalloc(&e->m_layer, sizeof(float) * n) == cudaSuccess &&
               cudaMalloc(&e->layer_gap, sizeof(float) * n) == cudaSuccess &&
               cudaMalloc(&e->layer_inv_gap, sizeof(float) * n) == cudaSuccess;
@@ -296,30 +303,53 @@ int build_layers(ga_engine* e, const int64_t* offsets, int n) {
     GA_CUDA(e, cudaMemset(e->m_layer, 0, sizeof(float) * n));
     GA_CUDA(e, cudaMemset(e->layer_gap, 0, sizeof(float) * n));
     GA_CUDA(e, cudaMemset(e->layer_ticket, 0, sizeof(unsigned int) * n));
+    GA_CUDA(e, cudaMemset(e->layer_epoch, 0, sizeof(unsigned int) * n));
+    e->layer_epoch_host = 0;
+
     e->layer_off.assign(offsets, offsets + n + 1);
     e->n_tiles = (int)nt;
     return GA_OK;
 }
 
-// Arrivals w.K of a window with the layer-wise Gap, one launch each. The Gap of the window's
-// first arrival is in place already when `primed` (the previous launch computed it); otherwise a
-// distance pass computes it first. `next_row` / `next_inv_bias` describe the arrival that follows
-// the window inside the same call (nullptr: none is known), so that the last launch of this window
-// can prepare its Gap as well.
+// A launch that may begin while the one before it on the stream is still draining (programmatic
+// dependent launch); the kernels order themselves through the layers' epoch counters.
+template <typename... Params, typename... Args>
+cudaError_t launch_chained(void (*kernel)(Params...), int grid, int block, cudaStream_t st, bool chained, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
+
+// Arrivals w.K of a window with the layer-wise Gap, one launch each, chained. The Gap of the
+// window's first arrival is in place already when `primed` (the launch before prepared it);
+// otherwise a distance pass computes it first. `next_row` / `next_inv_bias` describe the arrival
+// that follows the window inside the same call (nullptr: none is known), so that the window's last
+// arrival can prepare its Gap as well.
 int launch_layer_arrivals(ga_engine* e, const ga::Window& w, bool primed, const float* next_row, float next_inv_bias) {
     const ga::Hyper h = e->hyper();
     const ga::LayerTables T = e->layer_tables();
-    if (!primed)
-        ga::ga_layer_dist_kernel<<<e->n_tiles, ga::kLayerThreads, 0, e->stream>>>(e->theta, w.saved[0], T, w.inv_bias[0], h);
+    if (!primed) {   // opens a call: ordinary launch, after everything already on the stream
+        GA_CUDA(e, launch_chained(ga::ga_layer_dist_kernel, e->n_tiles, ga::kLayerThreads, e->stream, false, e->theta,
+                                  w.saved[0], T, w.inv_bias[0], h));
+        e->layer_epoch_host += 1;
+    }
     for (int j = 0; j < w.K; ++j) {
         const float* nxt = j + 1 < w.K ? w.saved[j + 1] : next_row;
         const float nxt_ib = j + 1 < w.K ? w.inv_bias[j + 1] : next_inv_bias;
         // the same worker again right away: its saved copy is the theta this launch writes, distance 0
         const int mode = !nxt ? 0 : (nxt == w.saved[j] && w.write_saved) ? 2 : 1;
-        ga::ga_layer_update_kernel<<<e->n_tiles, ga::kLayerThreads, 0, e->stream>>>(
-            e->theta, e->vel, w.grad[j], w.saved[j], w.write_saved, nxt, mode, T, e->lr, h, nxt_ib);
+        GA_CUDA(e, launch_chained(ga::ga_layer_arrival_kernel, e->n_tiles, ga::kLayerThreads, e->stream, true, e->theta,
+                                  e->vel, w.grad[j], w.saved[j], w.write_saved, nxt, mode, e->layer_epoch_host, T, e->lr, h,
+                                  nxt_ib, e->pull_err));
+        e->layer_epoch_host += 1;   // every arrival advances every layer's epoch once
     }
-    GA_CUDA(e, cudaGetLastError());
     return GA_OK;
 }
 
@@ -620,9 +650,10 @@ int ga_push_batch(ga_engine* e, const int* schedule_host, const float* const* gr
     int launches = 0;
     if (K > 0) e->stats_total = 0;
     if (e->is_layer()) {
-        // Arrivals are not fused in time (a layer's norm needs the whole vector between them), but
-        // each launch also measures the next arrival's distance: one launch per arrival after a
-        // first distance pass. The table is filled 16 arrivals at a time; a worker may repeat freely.
+        // A layer's norm needs the whole layer between arrivals, so they are not fused in time the way
+        // the parameter-wise kernel fuses them: one launch per arrival after a distance pass, chained
+        // so that each overlaps the tail of the one before (ga_layer_kernels.cuh). A worker may repeat
+        // freely; the table is filled 16 arrivals at a time.
         ga::Window cur, nxt;
         int n_cur = K < ga::kMaxWindow ? K : ga::kMaxWindow;
         if (K > 0) fill_window(e, cur, schedule_host, grads_host, n_cur, true, delays_out_host);
