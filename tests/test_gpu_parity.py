@@ -658,7 +658,7 @@ def test_single_arrival_against_fp64(P, math_mode):
         eng.close()
 
 
-@pytest.mark.parametrize("variant", ["GA", "DANA_GA", "ADAM_GA", "SA_GRAD", "GA_LAYER"])
+@pytest.mark.parametrize("variant", ["GA", "DANA_GA", "ADAM_GA", "ADAM_SA", "SA_GRAD", "GA_LAYER"])
 def test_extreme_values_round_like_the_oracle(P, variant):
     """States and gradients spanning the whole fp32 range -- subnormals, zeros of both signs,
     1e-42 .. 1e38, infinities, NaNs -- imported into both sides; a window of three arrivals must
@@ -690,7 +690,7 @@ def test_extreme_values_round_like_the_oracle(P, variant):
     extra = {}
     if variant == "DANA_GA":
         extra = dict(v_workers=np.stack([wild() for _ in range(n)]))
-    if variant == "ADAM_GA":
+    if variant.startswith("ADAM"):
         extra = dict(v_workers=wild(nonneg=True))
     o.set_state(theta, v, m, saved, iters, 5, 5, **extra)
     if variant == "GA_LAYER":                      # three layers; their m_p start at 0 on both sides
@@ -700,7 +700,7 @@ def test_extreme_values_round_like_the_oracle(P, variant):
     st.update(theta=theta, v=v, m=m, saved=saved, iter=iters, k_done=5, k_c=5)
     if variant == "DANA_GA":
         st["v_workers"] = extra["v_workers"]
-    if variant == "ADAM_GA":
+    if variant.startswith("ADAM"):
         st["v2"] = extra["v_workers"]
     eng.import_state(P.pack_state(st))
     grads = [wild() for _ in range(3)]
@@ -709,7 +709,7 @@ def test_extreme_values_round_like_the_oracle(P, variant):
     pairs = [(P.GA_THETA, o.get(o.THETA)), (P.GA_V, o.get(o.V))]
     if variant in ("GA", "DANA_GA", "ADAM_GA"):
         pairs.append((P.GA_M, o.get(o.M)))
-    if variant == "ADAM_GA":
+    if variant.startswith("ADAM"):
         pairs.append((P.GA_V2, o.second_moment()))
     for which, ref in pairs:
         got = _np(eng.get(which))

@@ -379,7 +379,7 @@ def test_short_exact_forms_agree_with_ieee_on_this_device(P):
     assert P.lib().ga_selftest_exact_forms(7, None) == P.GA_ERR_ARG
 
 
-@pytest.mark.parametrize("variant", ["GA", "DANA_GA", "ADAM_GA", "ADAM"])
+@pytest.mark.parametrize("variant", ["GA", "DANA_GA", "ADAM_GA", "ADAM", "ADAM_SA"])
 def test_short_forms_and_ieee_fallback_give_the_same_bits(P, variant):
     """The same three arrivals with hyper-parameters inside the proven ranges (short forms on) and
     from a checkpoint whose eta_max lies outside them (every element takes the IEEE routines): both
@@ -419,7 +419,7 @@ def test_short_forms_and_ieee_fallback_give_the_same_bits(P, variant):
         sched = [1, 0, 2]
         assert eng.push_batch(sched, [torch.from_numpy(g).cuda() for g in grads]) == o.push_batch(sched, grads)
         pairs = [(P.GA_THETA, o.get(o.THETA)), (P.GA_V, o.get(o.V))]
-        if variant != "ADAM":
+        if variant not in ("ADAM", "ADAM_SA"):
             pairs.append((P.GA_M, o.get(o.M)))
         if variant.startswith("ADAM"):
             pairs.append((P.GA_V2, o.second_moment()))
