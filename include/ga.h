@@ -243,8 +243,9 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len);
  *     over every divisor in [1, 2^100], and for tiny and subnormal distances;
  *   level 1 (about a minute): additionally the division for all 2^46 pairs of significands.
  * Returns the number of operands on which a short form differs from IEEE (0 on a B200), or a
- * negative GA_ERR_* code. Allocates 8 bytes of device memory for the duration of the call and
- * synchronises cuda_stream. */
+ * negative GA_ERR_* code (GA_ERR_STATE if the comparison fails to see a difference planted outside
+ * the ranges in use, where one is known to exist). Allocates 16 bytes of device memory for the
+ * duration of the call and synchronises cuda_stream. */
 int64_t ga_selftest_exact_forms(int level, void* cuda_stream);
 
 /* Gap statistics without any allocation. (The paper has no counterpart of this call; it exists

@@ -1024,9 +1024,9 @@ extern "C" int64_t ga_selftest_exact_forms(int level, void* cuda_stream) {
     if (level < 0 || level > 1) return fail(GA_ERR_ARG, "level must be 0 or 1");
     cudaStream_t st = (cudaStream_t)cuda_stream;
     unsigned long long* bad = nullptr;
-    if (cudaMalloc(&bad, sizeof *bad) != cudaSuccess) { cudaGetLastError(); return fail(GA_ERR_OOM, "cannot allocate a counter"); }
+    if (cudaMalloc(&bad, 2 * sizeof *bad) != cudaSuccess) { cudaGetLastError(); return fail(GA_ERR_OOM, "cannot allocate the counters"); }
     auto done = [&](int64_t rc) { cudaFree(bad); return rc; };
-    if (cudaMemsetAsync(bad, 0, sizeof *bad, st) != cudaSuccess) return done(fail(GA_ERR_CUDA, "cudaMemsetAsync failed"));
+    if (cudaMemsetAsync(bad, 0, 2 * sizeof *bad, st) != cudaSuccess) return done(fail(GA_ERR_CUDA, "cudaMemsetAsync failed"));
     namespace t = ga::selftest;
     const int grid = 148 * 16, block = 256;
     t::rcp_range<<<grid, block, 0, st>>>(0x0d800000u, 0x71800001u, bad);                 // every b in [2^-100, 2^100]
@@ -1038,12 +1038,16 @@ extern "C" int64_t ga_selftest_exact_forms(int level, void* cuda_stream) {
     t::gap_small_dist<<<grid, block, 0, st>>>(1u << 19, 4, bad);
     if (level >= 1)
         for (uint32_t slice = 0; slice < 64; ++slice) t::div_all_significands<<<1024, 128, 0, st>>>(slice << 17, bad);
-    unsigned long long host = 0;
+    // the comparison itself is checked too: beyond 2^126 the short reciprocal is known to differ from
+    // the IEEE one (its result would be subnormal), so the second counter must come back non-zero
+    t::rcp_range<<<4, block, 0, st>>>(0x7e800000u, 0x7e800400u, bad + 1);
+    unsigned long long host[2] = {0, 0};
     cudaError_t err = cudaGetLastError();
-    if (err == cudaSuccess) err = cudaMemcpyAsync(&host, bad, sizeof host, cudaMemcpyDeviceToHost, st);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(host, bad, sizeof host, cudaMemcpyDeviceToHost, st);
     if (err == cudaSuccess) err = cudaStreamSynchronize(st);
     if (err != cudaSuccess) return done(fail(GA_ERR_CUDA, "ga_selftest_exact_forms: %s", cudaGetErrorString(err)));
-    return done((int64_t)host);
+    if (host[1] == 0) return done(fail(GA_ERR_STATE, "the self-test did not see a difference where one is known to exist"));
+    return done((int64_t)host[0]);
 }
 
 // ============================================================ allocation-free Gap statistics
