@@ -248,6 +248,16 @@ int ga_import_state(ga_engine* e, const void* buf_host, size_t len);
  * duration of the call and synchronises cuda_stream. */
 int64_t ga_selftest_exact_forms(int level, void* cuda_stream);
 
+/* Self-test of the bounded waits. The layer-wise kernels (GA_GA_LAYER) order consecutive arrivals by
+ * waiting, layer by layer, for a counter that the previous arrival advances; like the bulk-copy waits
+ * of ga_pull these waits have an iteration limit, after which the block raises the engine's error
+ * flag and returns, and the engine reports GA_ERR_CUDA from its next synchronising call. This call
+ * launches one block that waits for a counter nothing advances and checks that the wait runs out
+ * (after about a second), that the flag is raised and that the kernel returns, leaving the
+ * context usable. Returns GA_OK, GA_ERR_STATE if the wait did not behave so, or another negative
+ * GA_ERR_* code. Allocates a few words for the duration of the call; synchronises cuda_stream. */
+int ga_selftest_bounded_wait(void* cuda_stream);
+
 /* Gap statistics without any allocation. (The paper has no counterpart of this call; it exists
  * for deployment reasons only.) Computes the sum and the maximum over all parameters of the
  * parameter-wise Gap |theta - saved| / C + 1, with C = lr_max * (sqrt(m / (1 - c_beta^n_refreshes))

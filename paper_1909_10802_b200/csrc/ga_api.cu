@@ -52,12 +52,13 @@ struct ga_engine {
     double* tile_partial = nullptr;   // 2 x n_tiles: sums of v^2, then sums of squared distances
     unsigned int* layer_ticket = nullptr;
     unsigned int* layer_epoch = nullptr;   // per layer: Gaps made ready so far; layer_epoch_host mirrors their common value
+    int* layer_abort = nullptr;            // device word: a wait of the layer kernels ran out
     unsigned int layer_epoch_host = 0;
     float *m_layer = nullptr, *layer_gap = nullptr, *layer_inv_gap = nullptr;
     int n_tiles = 0;
     ga::LayerTables layer_tables() const {
         return ga::LayerTables{tiles, tile_begin, tile_partial, tile_partial + n_tiles, layer_ticket, layer_epoch,
-                               m_layer, layer_gap, layer_inv_gap};
+                               layer_abort, m_layer, layer_gap, layer_inv_gap};
     }
     bool is_layer() const { return variant == GA_GA_LAYER; }
     int n_layers() const { return (int)layer_off.size() - 1; }
@@ -261,7 +262,9 @@ int launch_window(ga_engine* e, const ga::Window& w, long long vec_begin, long l
 void free_layers(ga_engine* e) {
     cudaFree(e->tiles); cudaFree(e->tile_begin); cudaFree(e->tile_partial); cudaFree(e->layer_ticket);
     cudaFree(e->layer_epoch);
+    cudaFree(e->layer_abort);
     e->layer_epoch = nullptr;
+    e->layer_abort = nullptr;
     cudaFree(e->m_layer); cudaFree(e->layer_gap); cudaFree(e->layer_inv_gap);
     e->tiles = nullptr; e->tile_begin = nullptr; e->tile_partial = nullptr; e->layer_ticket = nullptr;
     e->m_layer = e->layer_gap = e->layer_inv_gap = nullptr;
@@ -290,6 +293,7 @@ int build_layers(ga_engine* e, const int64_t* offsets, int n) {
               cudaMalloc(&e->tile_partial, sizeof(double) * 2 * nt) == cudaSuccess &&
               cudaMalloc(&e->layer_ticket, sizeof(unsigned int) * n) == cudaSuccess &&
               cudaMalloc(&e->layer_epoch, sizeof(unsigned int) * n) == cudaSuccess &&
+              cudaMalloc(&e->layer_abort, sizeof(int)) == cudaSuccess &&
               cudaMalloc(&e->m_layer, sizeof(float) * n) == cudaSuccess &&
               cudaMalloc(&e->layer_gap, sizeof(float) * n) == cudaSuccess &&
               cudaMalloc(&e->layer_inv_gap, sizeof(float) * n) == cudaSuccess;
@@ -304,6 +308,7 @@ int build_layers(ga_engine* e, const int64_t* offsets, int n) {
     GA_CUDA(e, cudaMemset(e->layer_gap, 0, sizeof(float) * n));
     GA_CUDA(e, cudaMemset(e->layer_ticket, 0, sizeof(unsigned int) * n));
     GA_CUDA(e, cudaMemset(e->layer_epoch, 0, sizeof(unsigned int) * n));
+    GA_CUDA(e, cudaMemset(e->layer_abort, 0, sizeof(int)));
     e->layer_epoch_host = 0;
 
     e->layer_off.assign(offsets, offsets + n + 1);
@@ -1048,6 +1053,38 @@ extern "C" int64_t ga_selftest_exact_forms(int level, void* cuda_stream) {
     if (err != cudaSuccess) return done(fail(GA_ERR_CUDA, "ga_selftest_exact_forms: %s", cudaGetErrorString(err)));
     if (host[1] == 0) return done(fail(GA_ERR_STATE, "the self-test did not see a difference where one is known to exist"));
     return done((int64_t)host[0]);
+}
+
+// A wait inside the layer-wise kernels that nothing satisfies: it has to give up and say so.
+extern "C" int ga_selftest_bounded_wait(void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    unsigned int* epoch = nullptr;   // epoch word, then the abort word
+    int* gave_up = nullptr;
+    int* flag = nullptr;   // mapped host memory, like an engine's error flag
+    int rc = GA_OK;
+    if (cudaMalloc(&epoch, 2 * sizeof *epoch) != cudaSuccess || cudaMalloc(&gave_up, sizeof *gave_up) != cudaSuccess ||
+        cudaHostAlloc(&flag, sizeof *flag, cudaHostAllocMapped) != cudaSuccess) {
+        cudaGetLastError();
+        rc = fail(GA_ERR_OOM, "cannot allocate the probe's words");
+    } else {
+        *flag = 0;
+        int host_gave_up = -1;
+        cudaError_t err = cudaMemsetAsync(epoch, 0, 2 * sizeof *epoch, st);
+        if (err == cudaSuccess) err = cudaMemsetAsync(gave_up, 0xff, sizeof *gave_up, st);
+        if (err == cudaSuccess) {
+            ga::ga_layer_wait_probe_kernel<<<1, ga::kLayerThreads, 0, st>>>(epoch, (int*)(epoch + 1), flag, gave_up);
+            err = cudaGetLastError();
+        }
+        if (err == cudaSuccess) err = cudaMemcpyAsync(&host_gave_up, gave_up, sizeof host_gave_up, cudaMemcpyDeviceToHost, st);
+        if (err == cudaSuccess) err = cudaStreamSynchronize(st);
+        if (err != cudaSuccess) rc = fail(GA_ERR_CUDA, "ga_selftest_bounded_wait: %s", cudaGetErrorString(err));
+        else if (host_gave_up != 1 || *(volatile int*)flag != 2)
+            rc = fail(GA_ERR_STATE, "the wait did not give up as it should (gave_up %d, flag %d)", host_gave_up, *flag);
+    }
+    cudaFree(epoch);
+    cudaFree(gave_up);
+    if (flag) cudaFreeHost(flag);
+    return rc;
 }
 
 // ============================================================ allocation-free Gap statistics

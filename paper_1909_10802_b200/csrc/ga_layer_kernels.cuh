@@ -53,6 +53,7 @@ struct LayerTables {
     double* partial_d;       // per tile: sum of (theta - saved copy)^2
     unsigned int* ticket;    // per layer, 0 between launches
     unsigned int* epoch;     // per layer: Gaps made ready so far (distance passes and arrivals), never reset
+    int* abort_word;         // set by a block whose wait ran out; ends every later wait at once
     float* m_layer;          // m_p of the C algorithm
     float* gap;              // G_p of the most recent arrival
     float* inv_gap;          // 1 / G_p of the arrival about to be applied
@@ -128,10 +129,13 @@ __device__ __forceinline__ void layer_gap(const LayerTables& T, int layer, doubl
     T.inv_gap[layer] = __frcp_rn(G);
 }
 
-constexpr unsigned kLayerSpinLimit = 1u << 22;   // polls of a layer's epoch before a block gives up
+constexpr unsigned kLayerSpinLimit = 1u << 20;   // polls of a layer's epoch (about a second) before a block gives up
 
 // Waits (thread 0 polls, everybody gets the answer) until the layer's epoch has reached `need`.
-__device__ __forceinline__ bool wait_layer_epoch(const unsigned int* epoch, unsigned int need, int* err) {
+// A block whose wait runs out raises the engine's error flag (mapped host memory) and a device-side
+// abort word, which every other waiting block sees at its next poll, so one lost dependency ends the
+// launches that follow in about a second instead of one time-out per block.
+__device__ __forceinline__ bool wait_layer_epoch(const unsigned int* epoch, unsigned int need, int* abort_word, int* err) {
     __shared__ int s_ready;
     if (threadIdx.x == 0) {
         int ready = 0;
@@ -139,9 +143,14 @@ __device__ __forceinline__ bool wait_layer_epoch(const unsigned int* epoch, unsi
             unsigned int seen;
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(epoch) : "memory");
             if ((int)(seen - need) >= 0) { ready = 1; break; }
+            if (*(volatile int*)abort_word) break;
             __nanosleep(64);
         }
-        if (!ready) { *(volatile int*)err = 2; __threadfence_system(); }   // mapped host memory
+        if (!ready) {
+            *(volatile int*)abort_word = 1;
+            *(volatile int*)err = 2;
+            __threadfence_system();
+        }
         s_ready = ready;
     }
     __syncthreads();
@@ -261,8 +270,16 @@ ga_layer_arrival_kernel(float* __restrict__ theta, float* __restrict__ vel, cons
                         unsigned int need, LayerTables T, float eta, const __grid_constant__ Hyper h, float inv_bias_next,
                         int* err) {
     release_dependent_launch();
-    if (!wait_layer_epoch(&T.epoch[T.tiles[blockIdx.x].layer], need, err)) return;
+    if (!wait_layer_epoch(&T.epoch[T.tiles[blockIdx.x].layer], need, T.abort_word, err)) return;
     update_tile(theta, vel, grad, saved, write_saved, next, next_mode, T, blockIdx.x, eta, h, inv_bias_next);
+}
+
+// One block that waits for an epoch nobody advances: the wait must run out, raise the flag and let the
+// block return (ga_selftest_bounded_wait).
+__global__ void __launch_bounds__(kLayerThreads)
+ga_layer_wait_probe_kernel(const unsigned int* epoch, int* abort_word, int* err, int* gave_up) {
+    const bool ready = wait_layer_epoch(epoch, 1u, abort_word, err);
+    if (threadIdx.x == 0) *gave_up = ready ? 0 : 1;
 }
 
 }  // namespace ga

@@ -428,3 +428,20 @@ def test_short_forms_and_ieee_fallback_give_the_same_bits(P, variant):
             bad = ~((got == ref.astype(np.float32)) | (np.isnan(got) & np.isnan(ref)))
             assert not bad.any(), (variant, lr_max, which, int(bad.sum()), got[bad][:4], ref[bad][:4])
         eng.close()
+
+
+# ----------------------------------------------------------------------------- bounded waits
+def test_a_wait_that_nothing_satisfies_gives_up_and_reports(P):
+    """The layer-wise kernels wait for per-layer counters; such a wait must end by itself. One block
+    waits for a counter nothing advances: the wait runs out, the error flag is raised, the kernel
+    returns and the context stays usable (a second engine runs right after)."""
+    import time
+    import torch
+    t0 = time.time()
+    assert P.lib().ga_selftest_bounded_wait(None) == P.GA_OK, P.last_error()
+    assert time.time() - t0 < 30.0
+    eng = P.Engine(1000, 2, 0.1, 0.9, 0.999, P.GA_GA_LAYER)
+    eng.set_params(torch.zeros(1000, device="cuda"))
+    assert eng.push_batch([0, 1], [torch.ones(1000, device="cuda")] * 2) == [1, 2]
+    assert torch.isfinite(eng.get(P.GA_THETA)).all()
+    eng.close()
