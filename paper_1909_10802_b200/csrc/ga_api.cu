@@ -74,6 +74,7 @@ struct ga_engine {
     ga::StatsPartial* partials = nullptr;
     double* stats_dev = nullptr;   // ring of kStatsLog x {sum, max}: one pair per arrival
     int stats_blocks = 0;
+    int small_range_vectors = 0;   // ranges of fewer 16-byte vectors than this run with two parameters per thread
     int64_t stats_total = 0;       // arrivals logged since the current call began (slot = index % kStatsLog)
     // pull kernel error flag: one int of pinned, device-mapped host memory
     int* pull_err = nullptr;
@@ -204,19 +205,26 @@ int grid_1d(long long n, int threads, int cap) {
 template <int FAMILY, int PENALTY, bool EXACT, int C_ORDER, bool STATS>
 void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, long long vec_end, cudaStream_t st,
                      int stats_mode) {
-    const long long nvec = vec_end - vec_begin;
-    long long blocks = (nvec + ga::kThreads - 1) / ga::kThreads;
+    // vec_begin / vec_end count 16-byte vectors (four parameters). A range too short to give every SM
+    // a full set of blocks at four parameters per thread runs with two per thread instead: twice the
+    // warps to hide an arrival's dependent chain behind, which is what bounds an L2-resident vector.
+    const bool narrow = (vec_end - vec_begin) < (long long)e->small_range_vectors;
+    const long long first = narrow ? vec_begin * 2 : vec_begin, last = narrow ? vec_end * 2 : vec_end;
+    long long blocks = (last - first + ga::kThreads - 1) / ga::kThreads;
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
     // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner.
     constexpr int ST = GA_WINDOW_STAGES;
-#define GA_LAUNCH(BATCH, STAGES_, WD_)                                                                          \
-    ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, BATCH, STAGES_, WD_>                            \
-        <<<(unsigned)blocks, ga::kThreads, 0, st>>>(e->theta, e->vel, e->mom, e->sec, w, e->hyper(), vec_begin, \
-                                                    vec_end, e->d, e->partials)
+#define GA_LAUNCH_V(BATCH, STAGES_, WD_, VEC_)                                                                   \
+    ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, BATCH, STAGES_, WD_, VEC_>                       \
+        <<<(unsigned)blocks, ga::kThreads, 0, st>>>(e->theta, e->vel, e->mom, e->sec, w, e->hyper(), first, last, \
+                                                    e->d, e->partials)
+#define GA_LAUNCH(BATCH, STAGES_, WD_) \
+    do { if (narrow) GA_LAUNCH_V(BATCH, STAGES_, WD_, 2); else GA_LAUNCH_V(BATCH, STAGES_, WD_, 4); } while (0)
     const bool wd = e->weight_decay != 0.f || e->nesterov;   // the instantiations with the extras
     if (w.K == 1) { if (wd) GA_LAUNCH(1, 0, true); else GA_LAUNCH(1, 0, false); }
     else { if (wd) GA_LAUNCH(GA_WINDOW_BATCH, ST, true); else GA_LAUNCH(GA_WINDOW_BATCH, ST, false); }
 #undef GA_LAUNCH
+#undef GA_LAUNCH_V
     if (STATS) {
         ga::ga_stats_finish_kernel<<<w.K, 256, 0, st>>>(e->partials, (int)blocks, e->stats_dev, e->stats_total,
                                                         kStatsLog, stats_mode == 2);
@@ -483,6 +491,7 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
     int sms = 148;
     if (cudaGetDeviceProperties(&prop, e->device) == cudaSuccess) sms = prop.multiProcessorCount;
     e->stats_blocks = sms * 8;
+    e->small_range_vectors = sms * 9 * ga::kThreads;   // one full set of resident blocks at four parameters per thread
     const size_t row_bytes = sizeof(float) * (size_t)e->stride;
     bool ok = cudaMalloc(&e->theta, row_bytes) == cudaSuccess && cudaMalloc(&e->vel, row_bytes) == cudaSuccess &&
               cudaMalloc(&e->mom, row_bytes) == cudaSuccess &&
