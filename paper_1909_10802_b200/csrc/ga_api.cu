@@ -31,7 +31,14 @@ int fail(int code, const char* fmt, ...) {
 }
 
 constexpr long long kRowAlign = 32;            // floats: rows start on 128-byte boundaries
-constexpr long long kHostChunk = 4ll << 20;    // floats per chunk of the host-buffer path
+#ifndef GA_HOST_CHUNK_FLOATS
+#define GA_HOST_CHUNK_FLOATS (4ll << 20)
+#endif
+#ifndef GA_HOST_STAGES
+#define GA_HOST_STAGES 2
+#endif
+constexpr long long kHostChunk = GA_HOST_CHUNK_FLOATS;   // floats per chunk of the host-buffer path
+constexpr int kHostStages = GA_HOST_STAGES;              // staging buffers the copies-in rotate through
 constexpr int kHostD2hRing = 4;                // chunks the kernels may run ahead of the copies out
 constexpr uint32_t kStateMagic = 0x47415331;   // "GAS1"
 constexpr int kStatsLog = GA_STATS_LOG;        // arrivals whose Gap statistics are kept
@@ -82,10 +89,10 @@ struct ga_engine {
     struct PowCache { double base = 0.0, p = 0.0; int64_t k = -1; };
     PowCache pow_c, pow_b1, pow_b2;
     // host-buffer path
-    float* stage[2] = {nullptr, nullptr};
+    float* stage[kHostStages] = {};
     long long stage_elems = 0;
     cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
-    cudaEvent_t ev_h2d[2] = {nullptr, nullptr}, ev_kernel[2] = {nullptr, nullptr}, ev_prev = nullptr;
+    cudaEvent_t ev_h2d[kHostStages] = {}, ev_kernel[kHostStages] = {}, ev_prev = nullptr;
     cudaEvent_t ev_d2h[kHostD2hRing] = {};
 
     float* row(int i) const { return saved + (size_t)i * stride; }
@@ -437,7 +444,7 @@ int ensure_host_path(ga_engine* e) {
     if (e->stage[0]) return GA_OK;
     const long long chunk = e->stride < kHostChunk ? e->stride : kHostChunk;
     e->stage_elems = chunk;
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < kHostStages; ++s) {
         if (cudaMalloc(&e->stage[s], sizeof(float) * (size_t)chunk * ga::kMaxWindow) != cudaSuccess) {
             cudaGetLastError();
             return fail(GA_ERR_OOM, "cannot allocate staging buffers for the host-buffer path");
@@ -539,7 +546,7 @@ void ga_destroy(ga_engine* e) {
     cudaFree(e->partials);
     cudaFree(e->stats_dev);
     cudaFreeHost(e->pull_err);
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < kHostStages; ++s) {
         cudaFree(e->stage[s]);
         if (e->ev_h2d[s]) cudaEventDestroy(e->ev_h2d[s]);
         if (e->ev_kernel[s]) cudaEventDestroy(e->ev_kernel[s]);
@@ -728,11 +735,11 @@ int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* cons
         const float* staged[ga::kMaxWindow] = {};
         fill_window(e, w, schedule_host + pos, staged, n, true, delays_out_host ? delays_out_host + pos : nullptr);
         for (long long c0 = 0, c = 0; c0 < e->stride; c0 += chunk, ++c, ++g) {
-            const int s = (int)(g & 1);
+            const int s = (int)(g % kHostStages);
             const long long c1 = c0 + chunk < e->stride ? c0 + chunk : e->stride;
             const long long valid = (c1 < e->d ? c1 : e->d) - c0;   // floats the caller's buffers hold
-            // staging buffer s is free once the kernel that read it two chunks ago has run
-            if (g >= 2) GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_kernel[s], 0));
+            // staging buffer s is free once the kernel that read it kHostStages chunks ago has run
+            if (g >= kHostStages) GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_kernel[s], 0));
             for (int j = 0; j < n; ++j) {
                 float* dst = e->stage[s] + (size_t)j * chunk;
                 if (valid > 0)
