@@ -115,6 +115,20 @@ enum {
 ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, float c_beta,
                      int variant);
 
+/* The same master inside memory the caller provides: for processes in which a framework's
+ * allocator owns the device memory (the state of a master is large -- Appendix "Gap-Aware Overhead":
+ * one copy of the parameters per worker -- and should then come out of that pool, not compete with
+ * it). ga_workspace_bytes returns the size needed for theta, v, m, the n_workers saved copies, the
+ * DANA variants' per-worker momentum vectors, Adam's second moment and the statistics buffers
+ * (0 on invalid arguments); ga_create_in lays them out in workspace_dev (device memory, 256-byte
+ * aligned, at least that many bytes, owned by the caller and kept alive and untouched until
+ * ga_destroy, which does not free it). Everything else is as for ga_create. Still allocated by the
+ * library itself: one word of pinned host memory per engine, the small per-layer tables of
+ * GA_GA_LAYER (ga_set_layers) and the staging buffers of ga_push_batch_host on its first use. */
+size_t ga_workspace_bytes(size_t n_params, int n_workers, int variant);
+ga_engine* ga_create_in(size_t n_params, int n_workers, float lr, float momentum, float c_beta,
+                        int variant, void* workspace_dev, size_t workspace_bytes);
+
 /* Free everything the engine owns. NULL is accepted. Synchronises the bound stream first. */
 void ga_destroy(ga_engine* e);
 

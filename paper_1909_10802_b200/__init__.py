@@ -32,6 +32,9 @@ VARIANTS = {"ASGD": GA_ASGD, "SA": GA_SA, "GA": GA_GA, "SA_GRAD": GA_SA_GRAD, "D
 _c = ctypes
 _SIGNATURES = {
     "ga_create": (_c.c_void_p, [_c.c_size_t, _c.c_int, _c.c_float, _c.c_float, _c.c_float, _c.c_int]),
+    "ga_workspace_bytes": (_c.c_size_t, [_c.c_size_t, _c.c_int, _c.c_int]),
+    "ga_create_in": (_c.c_void_p, [_c.c_size_t, _c.c_int, _c.c_float, _c.c_float, _c.c_float, _c.c_int, _c.c_void_p,
+                                   _c.c_size_t]),
     "ga_destroy": (None, [_c.c_void_p]),
     "ga_set_stream": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
     "ga_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
@@ -118,6 +121,16 @@ def gap_stats_noalloc(theta, saved, m, lr_max, c_beta, n_refreshes, out, stream=
     return out
 
 
+def workspace_bytes(n_params, n_workers, variant=GA_GA):
+    """ga_workspace_bytes: device bytes an Engine(..., workspace=...) of this shape needs."""
+    if isinstance(variant, str):
+        variant = VARIANTS[variant]
+    n = lib().ga_workspace_bytes(int(n_params), int(n_workers), variant)
+    if n == 0:
+        raise GaError(GA_ERR_ARG, last_error())
+    return n
+
+
 def selftest_exact_forms(level=0, stream=None):
     """ga_selftest_exact_forms: operands on which the kernels' short exact forms differ from the
     IEEE routines on the current device (0 = they agree everywhere they are used)."""
@@ -130,7 +143,9 @@ class Engine:
     """One master. Thin wrapper: methods carry the names of the C calls without the prefix."""
 
     def __init__(self, n_params, n_workers, lr=0.1, momentum=0.9, c_beta=0.999, variant=GA_GA,
-                 stream=None):
+                 stream=None, workspace=None):
+        """workspace: a CUDA tensor (any dtype) of at least workspace_bytes(...) bytes in which the
+        engine keeps its state (ga_create_in); the engine holds a reference to it."""
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("the Gap-Aware master needs a CUDA device; there is no CPU path")
@@ -141,7 +156,13 @@ class Engine:
         self.n_params, self.n_workers, self.variant = int(n_params), int(n_workers), variant
         torch.cuda.init()
         torch.zeros(1, device="cuda")      # make sure a context exists on the current device
-        self._h = self._l.ga_create(self.n_params, self.n_workers, lr, momentum, c_beta, variant)
+        self._workspace = workspace
+        if workspace is None:
+            self._h = self._l.ga_create(self.n_params, self.n_workers, lr, momentum, c_beta, variant)
+        else:
+            assert workspace.is_cuda and workspace.is_contiguous()
+            self._h = self._l.ga_create_in(self.n_params, self.n_workers, lr, momentum, c_beta, variant,
+                                           workspace.data_ptr(), workspace.numel() * workspace.element_size())
         if not self._h:
             raise GaError(GA_ERR_ARG, last_error())
         self.set_stream(stream if stream is not None else torch.cuda.current_stream())

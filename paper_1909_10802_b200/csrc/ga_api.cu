@@ -77,6 +77,7 @@ struct ga_engine {
     int64_t k_done = 0, k_c = 0;
     cudaStream_t stream = nullptr;
     bool cuda_failed = false;
+    bool owns_state = true;        // false: theta, v, m, the copies and the statistics buffers live in the caller's workspace
     // statistics
     ga::StatsPartial* partials = nullptr;
     double* stats_dev = nullptr;   // ring of kStatsLog x {sum, max}: one pair per arrival
@@ -466,7 +467,42 @@ extern "C" {
 
 const char* ga_last_error(void) { return g_error.c_str(); }
 
-ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, float c_beta, int variant) {
+}  // extern "C"
+
+namespace {
+
+constexpr int kMaxStatsBlocks = 2048;   // the workspace reserves room for this many per-block partials per arrival
+
+bool is_dana_variant(int v) { return v == GA_DANA || v == GA_DANA_SA || v == GA_DANA_GA; }
+bool is_adam_variant(int v) { return v == GA_ADAM || v == GA_ADAM_SA || v == GA_ADAM_GA; }
+
+// Where everything of fixed size lives inside one device allocation (offsets in bytes, 256-byte aligned).
+struct StatePlan {
+    size_t theta, vel, mom, saved, vworker, sec, partials, stats, total;
+};
+
+StatePlan plan_state(long long stride, int n_workers, int variant) {
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    const size_t row = up(sizeof(float) * (size_t)stride);   // rows are multiples of 128 bytes already
+    StatePlan p{};
+    size_t at = 0;
+    p.theta = at; at += row;
+    p.vel = at; at += row;
+    p.mom = at; at += row;
+    p.saved = at; at += up(sizeof(float) * (size_t)stride * (size_t)n_workers);
+    p.vworker = at; if (is_dana_variant(variant)) at += up(sizeof(float) * (size_t)stride * (size_t)n_workers);
+    p.sec = at; if (is_adam_variant(variant)) at += row;
+    p.partials = at; at += up(sizeof(ga::StatsPartial) * (size_t)kMaxStatsBlocks * ga::kMaxWindow);
+    p.stats = at; at += up(sizeof(double) * 2 * kStatsLog);
+    p.total = at;
+    return p;
+}
+
+long long padded_stride(size_t n_params) { return ((long long)n_params + kRowAlign - 1) / kRowAlign * kRowAlign; }
+
+// ga_create and ga_create_in: workspace == nullptr lets the engine allocate its own state.
+ga_engine* create_engine(size_t n_params, int n_workers, float lr, float momentum, float c_beta, int variant,
+                         void* workspace, size_t workspace_bytes, bool in_workspace) {
     g_error.clear();
     if (n_params == 0 || n_params > (size_t)1 << 34) { fail(GA_ERR_ARG, "n_params out of range"); return nullptr; }
     if (n_workers <= 0 || n_workers > 65536) { fail(GA_ERR_ARG, "n_workers out of range"); return nullptr; }
@@ -497,17 +533,38 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
     cudaDeviceProp prop;
     int sms = 148;
     if (cudaGetDeviceProperties(&prop, e->device) == cudaSuccess) sms = prop.multiProcessorCount;
-    e->stats_blocks = sms * 8;
+    e->stats_blocks = sms * 8 < kMaxStatsBlocks ? sms * 8 : kMaxStatsBlocks;
     e->small_range_vectors = sms * 9 * ga::kThreads;   // one full set of resident blocks at four parameters per thread
     const size_t row_bytes = sizeof(float) * (size_t)e->stride;
-    bool ok = cudaMalloc(&e->theta, row_bytes) == cudaSuccess && cudaMalloc(&e->vel, row_bytes) == cudaSuccess &&
-              cudaMalloc(&e->mom, row_bytes) == cudaSuccess &&
-              cudaMalloc(&e->saved, row_bytes * (size_t)n_workers) == cudaSuccess &&
-              cudaMalloc(&e->partials, sizeof(ga::StatsPartial) * (size_t)e->stats_blocks * ga::kMaxWindow) == cudaSuccess &&
-              cudaMalloc(&e->stats_dev, sizeof(double) * 2 * kStatsLog) == cudaSuccess &&
-              cudaHostAlloc(&e->pull_err, sizeof(int), cudaHostAllocMapped) == cudaSuccess &&
-              (!e->is_dana() || cudaMalloc(&e->vworker, row_bytes * (size_t)n_workers) == cudaSuccess) &&
-              (!e->is_adam() || cudaMalloc(&e->sec, row_bytes) == cudaSuccess);
+    bool ok;
+    if (in_workspace) {   // carve the caller's memory; nothing of it is ever freed here
+        const StatePlan p = plan_state(e->stride, n_workers, variant);
+        if (!workspace || (uintptr_t)workspace % 256 || workspace_bytes < p.total) {
+            fail(GA_ERR_ARG, "workspace must be 256-byte aligned device memory of at least %zu bytes (ga_workspace_bytes)", p.total);
+            delete e;
+            return nullptr;
+        }
+        char* base = (char*)workspace;
+        e->owns_state = false;
+        e->theta = (float*)(base + p.theta);
+        e->vel = (float*)(base + p.vel);
+        e->mom = (float*)(base + p.mom);
+        e->saved = (float*)(base + p.saved);
+        if (e->is_dana()) e->vworker = (float*)(base + p.vworker);
+        if (e->is_adam()) e->sec = (float*)(base + p.sec);
+        e->partials = (ga::StatsPartial*)(base + p.partials);
+        e->stats_dev = (double*)(base + p.stats);
+        ok = cudaHostAlloc(&e->pull_err, sizeof(int), cudaHostAllocMapped) == cudaSuccess;
+    } else {
+        ok = cudaMalloc(&e->theta, row_bytes) == cudaSuccess && cudaMalloc(&e->vel, row_bytes) == cudaSuccess &&
+             cudaMalloc(&e->mom, row_bytes) == cudaSuccess &&
+             cudaMalloc(&e->saved, row_bytes * (size_t)n_workers) == cudaSuccess &&
+             cudaMalloc(&e->partials, sizeof(ga::StatsPartial) * (size_t)e->stats_blocks * ga::kMaxWindow) == cudaSuccess &&
+             cudaMalloc(&e->stats_dev, sizeof(double) * 2 * kStatsLog) == cudaSuccess &&
+             cudaHostAlloc(&e->pull_err, sizeof(int), cudaHostAllocMapped) == cudaSuccess &&
+             (!e->is_dana() || cudaMalloc(&e->vworker, row_bytes * (size_t)n_workers) == cudaSuccess) &&
+             (!e->is_adam() || cudaMalloc(&e->sec, row_bytes) == cudaSuccess);
+    }
     if (ok) {
         ok = cudaMemset(e->theta, 0, row_bytes) == cudaSuccess && cudaMemset(e->vel, 0, row_bytes) == cudaSuccess &&
              cudaMemset(e->mom, 0, row_bytes) == cudaSuccess &&
@@ -532,19 +589,43 @@ ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, f
     return e;
 }
 
+}  // namespace
+
+extern "C" {
+
+ga_engine* ga_create(size_t n_params, int n_workers, float lr, float momentum, float c_beta, int variant) {
+    return create_engine(n_params, n_workers, lr, momentum, c_beta, variant, nullptr, 0, false);
+}
+
+size_t ga_workspace_bytes(size_t n_params, int n_workers, int variant) {
+    if (n_params == 0 || n_params > (size_t)1 << 34 || n_workers <= 0 || n_workers > 65536 || variant < GA_ASGD ||
+        variant > GA_GA_LAYER) {
+        fail(GA_ERR_ARG, "ga_workspace_bytes: arguments out of range");
+        return 0;
+    }
+    return plan_state(padded_stride(n_params), n_workers, variant).total;
+}
+
+ga_engine* ga_create_in(size_t n_params, int n_workers, float lr, float momentum, float c_beta, int variant,
+                        void* workspace_dev, size_t workspace_bytes) {
+    return create_engine(n_params, n_workers, lr, momentum, c_beta, variant, workspace_dev, workspace_bytes, true);
+}
+
 void ga_destroy(ga_engine* e) {
     if (!e) return;
     DeviceGuard guard(e->device);
     cudaStreamSynchronize(e->stream);
-    cudaFree(e->theta);
-    cudaFree(e->vel);
-    cudaFree(e->mom);
-    cudaFree(e->saved);
-    cudaFree(e->vworker);
-    cudaFree(e->sec);
+    if (e->owns_state) {
+        cudaFree(e->theta);
+        cudaFree(e->vel);
+        cudaFree(e->mom);
+        cudaFree(e->saved);
+        cudaFree(e->vworker);
+        cudaFree(e->sec);
+        cudaFree(e->partials);
+        cudaFree(e->stats_dev);
+    }
     free_layers(e);
-    cudaFree(e->partials);
-    cudaFree(e->stats_dev);
     cudaFreeHost(e->pull_err);
     for (int s = 0; s < kHostStages; ++s) {
         cudaFree(e->stage[s]);

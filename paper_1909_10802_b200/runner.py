@@ -13,7 +13,7 @@ from . import Engine, GA_MAX_WINDOW, GA_OPT_WINDOW, VARIANTS
 
 class Run:
     def __init__(self, wl, variant="GA", window=GA_MAX_WINDOW, options=None, torch_device="cuda",
-                 shard=None):
+                 shard=None, workspace=None):
         """shard = (j0, n): this engine holds parameters [j0, j0+n) of the workload's vector
         (every step is independent per parameter, so ranks need no exchange)."""
         import torch
@@ -22,7 +22,8 @@ class Run:
         self.j0, self.n = shard if shard is not None else (0, wl.d)
         self.dev = wl.device(torch_device, self.j0, self.n)
         self.window = window
-        self.engine = Engine(self.n, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, VARIANTS[variant])
+        self.engine = Engine(self.n, wl.n_workers, wl.lr, wl.momentum, wl.c_beta, VARIANTS[variant],
+                             workspace=workspace)    # workspace: a CUDA tensor that holds the engine's state
         self.engine.set_option(GA_OPT_WINDOW, window)
         if variant == "GA_LAYER":          # the workload's tensors are the layers
             assert shard is None, "a layer's norm needs the whole layer on one rank"

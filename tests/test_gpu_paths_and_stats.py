@@ -445,3 +445,47 @@ def test_a_wait_that_nothing_satisfies_gives_up_and_reports(P):
     assert eng.push_batch([0, 1], [torch.ones(1000, device="cuda")] * 2) == [1, 2]
     assert torch.isfinite(eng.get(P.GA_THETA)).all()
     eng.close()
+
+
+# ----------------------------------------------------------------------------- caller-owned memory
+@pytest.mark.parametrize("variant", ["GA", "DANA_GA", "ADAM_GA", "GA_LAYER"])
+def test_engine_inside_a_callers_workspace(P, variant):
+    """ga_create_in: the engine's state laid out in a torch tensor must behave exactly like an
+    engine that allocated for itself (oracle parity, statistics), must not write outside the bytes
+    ga_workspace_bytes asked for, and must leave the tensor alone after ga_destroy."""
+    import torch
+    from paper_1909_10802_b200.runner import Run
+    wl = W.config("mini")
+    need = P.workspace_bytes(wl.d, wl.n_workers, variant)
+    state_floats = wl.d * (3 + wl.n_workers * (2 if variant == "DANA_GA" else 1) + (1 if variant == "ADAM_GA" else 0))
+    assert 4 * state_floats < need < 4 * state_floats + (2 << 20)
+    pad = 4096
+    ws = torch.full((need + 2 * pad,), 0x5A, dtype=torch.uint8, device="cuda")
+    inner = ws[pad:pad + need]
+    assert inner.data_ptr() % 256 == 0
+
+    run = Run(wl, variant, 16, options={P.GA_OPT_STATS: 1} if variant != "GA_LAYER" else None, workspace=inner)
+    delays = run.run()
+    o, odelays, _ = run_oracle(wl, variant)
+    assert delays == odelays
+    for which, ow in ((P.GA_THETA, o.THETA), (P.GA_V, o.V)):
+        assert np.array_equal(_np(run.engine.get(which)), o.get(ow).astype(np.float32), equal_nan=True)
+    for i in range(wl.n_workers):
+        assert np.array_equal(_np(run.engine.saved(i)), o.saved(i).astype(np.float32), equal_nan=True)
+    if variant != "GA_LAYER":
+        s, m = run.engine.get_stats()
+        assert abs(s - o.stats()[0]) <= 1e-9 * o.stats()[0] and m == o.stats()[1]
+    theta_addr = run.engine.saved_ptr(0)
+    assert inner.data_ptr() <= theta_addr < inner.data_ptr() + need          # the copies live in the tensor
+    assert bool((ws[:pad] == 0x5A).all()) and bool((ws[pad + need:] == 0x5A).all())
+    run.close()
+    snapshot = ws.clone()
+    torch.cuda.synchronize()
+    assert torch.equal(ws, snapshot)
+    # too small, misaligned or missing workspaces are refused
+    l = P.lib()
+    assert not l.ga_create_in(wl.d, wl.n_workers, 0.1, 0.9, 0.999, P.VARIANTS[variant], inner.data_ptr(), need - 1)
+    assert "ga_workspace_bytes" in P.last_error()
+    assert not l.ga_create_in(wl.d, wl.n_workers, 0.1, 0.9, 0.999, P.VARIANTS[variant], inner.data_ptr() + 16, need)
+    assert not l.ga_create_in(wl.d, wl.n_workers, 0.1, 0.9, 0.999, P.VARIANTS[variant], None, need)
+    assert l.ga_workspace_bytes(0, 4, P.GA_GA) == 0
