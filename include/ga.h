@@ -87,7 +87,9 @@ enum {
                            and the maximum of the Gap over all parameters (the average Gap is what
                            Appendix "Gap and Delay" logs); read with ga_get_stats_window or
                            ga_get_stats. Default 0. Not computed for GA_GA_LAYER, which has one Gap
-                           per layer (see ga_get_layer_state). */
+                           per layer (see ga_get_layer_state). Non-finite values propagate by IEEE
+                           rules and nothing traps; with this option on they are also noticed: the
+                           sum of an arrival is NaN or infinite exactly when some parameter's Gap was. */
     GA_OPT_WINDOW = 3,  /* 1..16 (default 16): most arrivals fused into one launch by
                            ga_push_batch. */
     GA_OPT_ADAM_BETA2 = 4, /* Adam variants: beta_2 in [0,1), default 0.999; before the first arrival */

@@ -49,6 +49,10 @@ int main(void) {
     EXPECT(ga_gap_stats_noalloc(fake, fake, fake, 16, 0.1f, 1.0f, 1, out, NULL) == GA_ERR_ARG);
     EXPECT(ga_gap_stats_noalloc(fake, fake, fake, 16, 0.1f, 0.999f, -1, out, NULL) == GA_ERR_ARG);
 
+    EXPECT(ga_workspace_bytes(0, 3, GA_GA) == 0 && ga_workspace_bytes(10, 0, GA_GA) == 0 && ga_workspace_bytes(10, 3, 99) == 0);
+    EXPECT(ga_workspace_bytes(1000, 3, GA_DANA_GA) > ga_workspace_bytes(1000, 3, GA_GA));
+    EXPECT(ga_create_in(0, 3, 0.1f, 0.9f, 0.999f, GA_GA, fake, 1 << 20) == NULL);
+
     ga_engine* e = ga_create(1000, 3, 0.1f, 0.9f, 0.999f, GA_GA);
     if (!e) {   /* no CUDA device here: that must be an error message, not a crash */
         EXPECT(strlen(ga_last_error()) > 0);

@@ -489,3 +489,26 @@ def test_engine_inside_a_callers_workspace(P, variant):
     assert not l.ga_create_in(wl.d, wl.n_workers, 0.1, 0.9, 0.999, P.VARIANTS[variant], inner.data_ptr() + 16, need)
     assert not l.ga_create_in(wl.d, wl.n_workers, 0.1, 0.9, 0.999, P.VARIANTS[variant], None, need)
     assert l.ga_workspace_bytes(0, 4, P.GA_GA) == 0
+
+
+def test_statistics_notice_non_finite_values(P):
+    """Nothing traps on a diverged run; with GA_OPT_STATS the sum of the Gap turns non-finite as soon
+    as one parameter's Gap does (here: a NaN gradient poisons theta, so the next Gap taken against
+    that theta is NaN)."""
+    import math
+    import torch
+    d = 3000
+    eng = P.Engine(d, 2, 0.1, 0.9, 0.999, P.GA_GA)
+    eng.set_option(P.GA_OPT_STATS, 1)
+    eng.set_params(torch.zeros(d, device="cuda"))
+    g = torch.full((d,), 0.01, device="cuda")
+    eng.push_batch([0, 1], [g, g])
+    assert all(math.isfinite(s) for s, _ in eng.get_stats_window())
+    bad = g.clone()
+    bad[1234] = float("nan")
+    eng.push_batch([0], [bad])                 # theta[1234] becomes NaN
+    eng.push_batch([1], [g])                   # worker 1's Gap at 1234 is |NaN - s| / C + 1
+    (s, _), = eng.get_stats_window()
+    assert math.isnan(s)
+    assert int(torch.isnan(eng.get(P.GA_THETA)).sum()) == 1
+    eng.close()
