@@ -512,3 +512,41 @@ def test_statistics_notice_non_finite_values(P):
     assert math.isnan(s)
     assert int(torch.isnan(eng.get(P.GA_THETA)).sum()) == 1
     eng.close()
+
+
+def test_layer_gap_one_long_call(P):
+    """One ga_push_batch call of 45 arrivals with the layer-wise Gap: the call spans three arrival
+    tables of 16, so the second and third run 'primed' (their first Gap was prepared by the launch
+    before), workers repeat back to back (distance exactly 0) and at random. Every launch is
+    chained to the one before; the result must still equal the oracle's bit for bit."""
+    import torch
+    d, n = 50_003, 4
+    offsets = [0, 7, 4_100, 4_101, 30_000, d]
+    rng = np.random.default_rng(21)
+    th0 = rng.normal(size=d).astype(np.float32)
+    pool = [(0.1 * rng.normal(size=d)).astype(np.float32) for _ in range(5)]
+    sched = [int(x) for x in rng.integers(0, n, size=45)]
+    sched[10] = sched[11] = sched[12] = 2          # the same worker three times in a row
+    sched[15] = sched[16] = 1                      # ... and across the boundary of two tables
+    grads = [pool[k % 5] for k in range(len(sched))]
+    o = oracle.Oracle(d, n, 0.05, 0.9, 0.999, oracle.GA_LAYER)
+    o.set_layers(offsets)
+    o.set_params(th0)
+    eng = P.Engine(d, n, 0.05, 0.9, 0.999, P.GA_GA_LAYER)
+    eng.set_layers(offsets)
+    eng.set_params(torch.from_numpy(th0).cuda())
+    dev = [torch.from_numpy(g).cuda() for g in pool]
+    delays, launches = eng.push_batch(sched, [dev[k % 5] for k in range(len(sched))], return_launches=True)
+    assert delays == o.push_batch(sched, grads) and launches == len(sched) + 1
+    assert np.array_equal(_np(eng.get(P.GA_THETA)), o.get(o.THETA).astype(np.float32))
+    assert np.array_equal(_np(eng.get(P.GA_V)), o.get(o.V).astype(np.float32))
+    gaps, m_layer = eng.get_layer_state()
+    ogaps, om = o.layer_state()
+    assert np.array_equal(gaps, ogaps.astype(np.float32)) and np.array_equal(m_layer, om.astype(np.float32))
+    for i in range(n):
+        assert np.array_equal(_np(eng.saved(i)), o.saved(i).astype(np.float32))
+    # a second call continues from there (its distance pass runs after the chain has drained)
+    more = [3, 3, 0]
+    assert eng.push_batch(more, dev[:3]) == o.push_batch(more, pool[:3])
+    assert np.array_equal(_np(eng.get(P.GA_THETA)), o.get(o.THETA).astype(np.float32))
+    eng.close()
