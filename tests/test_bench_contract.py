@@ -24,6 +24,7 @@ def test_reference_arm_times_the_oracle():
     j = _run("--impl", "reference", "--params", "200000", "--workers", "8", "--steps", "2", "--warmup", "1")
     assert BASE_KEYS <= set(j) and j["impl"] == "reference" and j["value"] > 0
     assert j["cpu_baseline"]["kind"] == "oracle" and j["cpu_baseline"]["cores"] == 1
+    assert j["cpu_baseline"]["host_cores"] >= 1 and j["cpu_baseline"]["cpu_model"]
     assert j["e2e"] == {"value": j["value"], "unit": j["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert j["metric"] == "ga_master_param_updates_per_sec" and j["higher_is_better"] is True
 
@@ -45,3 +46,25 @@ def test_gpu_arm_small_case():
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert j["e2e"]["h2d_bytes_per_step"] > 0 and j["e2e"]["d2h_bytes_per_step"] > 0 and j["e2e"]["value"] > 0
     assert j["cpu_baseline"]["value"] > 0 and "workload" in j["config"]
+    cb = j["cpu_baseline"]
+    assert cb["cores"] == 1 and cb["host_cores"] >= 1 and isinstance(cb["cpu_model"], str)
+    assert "all_cores" in cb and (cb["all_cores"].get("value", 0) > 0 or "unavailable" in cb["all_cores"])
+    assert 0 < j["e2e"]["pcie_frac"] < 1.5 and j["e2e"]["pcie_h2d_gbs"] > 0 and j["e2e"]["pcie_d2h_gbs"] > 0
+    assert "traffic" in r and "traffic_source" in r     # a capture exists for GA / 16 / exact only while the kernel is unchanged
+
+
+def test_traffic_file_matches_the_kernel_source():
+    """roofline.traffic comes from profiles/ga_window_kernel_dram_traffic.json; the figure is only
+    reported while the kernel source has the digest recorded at capture time."""
+    sys.path.insert(0, ROOT)
+    import bench
+    value, source = bench.measured_traffic("GA", 16, "exact")
+    table = json.load(open(bench.TRAFFIC_FILE))
+    entry = table["captures"]["GA/16/exact"]
+    import hashlib
+    digest = hashlib.sha256(open(bench.KERNEL_SOURCE, "rb").read()).hexdigest()
+    if digest == entry["kernel_source_sha256"]:
+        assert value == entry["dram_bytes_per_param"] and 0.9 < value / entry["algorithmic_bytes_per_param"] < 1.1
+    else:
+        assert value is None and "changed" in source
+    assert bench.measured_traffic("SA", 16, "exact")[0] is None
