@@ -550,3 +550,35 @@ def test_layer_gap_one_long_call(P):
     assert eng.push_batch(more, dev[:3]) == o.push_batch(more, pool[:3])
     assert np.array_equal(_np(eng.get(P.GA_THETA)), o.get(o.THETA).astype(np.float32))
     eng.close()
+
+
+@pytest.mark.parametrize("variant", ["GA", "ADAM_GA"])
+def test_host_buffer_path_on_a_short_vector(P, variant):
+    """The host-buffer path on a vector short enough for the two-parameters-per-thread layout (one
+    chunk, ragged end), statistics on: equal to the device path and to the oracle."""
+    import torch
+    d, n = 10_007, 3
+    rng = np.random.default_rng(8)
+    th0 = rng.normal(size=d).astype(np.float32)
+    sched = [1, 0, 2, 0]
+    grads = [(0.1 * rng.normal(size=d)).astype(np.float32) for _ in sched]
+    var = P.VARIANTS[variant]
+    lr = 0.01 if variant == "ADAM_GA" else 0.1
+    o = oracle.Oracle(d, n, lr, 0.9, 0.999, oracle.VARIANTS[variant])
+    o.set_params(th0)
+    want = []
+    for i, g in zip(sched, grads):
+        o.push(i, g)
+        want.append(o.stats())
+        o.pull(i)
+    eng = P.Engine(d, n, lr, 0.9, 0.999, var)
+    eng.set_option(P.GA_OPT_STATS, 1)
+    eng.set_params(torch.from_numpy(th0).cuda())
+    outs = [torch.empty(d, dtype=torch.float32).pin_memory() for _ in sched]
+    eng.push_batch_host(sched, [torch.from_numpy(g).pin_memory() for g in grads], outs)
+    assert np.array_equal(_np(eng.get(P.GA_THETA)), o.get(o.THETA).astype(np.float32))
+    assert np.array_equal(_np(eng.get(P.GA_M)), o.get(o.M).astype(np.float32))
+    assert np.array_equal(outs[-1].numpy(), o.saved(0).astype(np.float32))
+    for (s, m), (os_, om) in zip(eng.get_stats_window(), want):
+        assert abs(s - os_) <= 1e-9 * os_ and m == om
+    eng.close()
