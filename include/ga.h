@@ -60,9 +60,11 @@ enum {
     /* Gap-Aware with the layer-wise Gap of Section 5.3: G_p = ||theta_p - theta^i_p|| / C_p + 1, one
      * number per layer (ga_set_layers); with a single layer -- the default -- it is the global Gap
      * of Definition 1. C_p comes from the C algorithm run on the squared norm of the layer's
-     * update vector. Norms are accumulated in fp64 and rounded to fp32 once. Each arrival takes
-     * two passes over the vector (the norm must be known before the update), so arrivals are not
-     * fused in time and ga_push_batch_host is not available for this variant. */
+     * update vector. Norms are accumulated in fp64 and rounded to fp32 once. A layer's norm must be
+     * known before the layer is updated, so arrivals are not fused in time: each is one launch over
+     * the vector, which inside a ga_push_batch call also measures the next arrival's distance (one
+     * extra distance pass per call), and consecutive launches overlap. ga_push_batch_host is not
+     * available for this variant. */
     GA_GA_LAYER = 10
 };
 
