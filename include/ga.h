@@ -80,11 +80,14 @@ enum {
                            k-1, and m is then refreshed with the master's new v. 1: "Adam order":
                            m is first refreshed with (gamma v + g)^2 of the raw gradient (the
                            printed line of the C algorithm), then C, Gap and the step follow. */
-    GA_OPT_MATH = 1,    /* 0 (default): every operation IEEE round-to-nearest, in the order of
-                           the algorithms. 1: fast: approximate reciprocal and square root, one
-                           division per element (g*C/(|theta-theta^i|+C)); a few ulp off. Applies
-                           to GA_GA, GA_DANA_GA and GA_ADAM_GA (there also to Adam's own root and
-                           division); every other variant is always exact. */
+    GA_OPT_MATH = 1,    /* 0 (default): exact -- every symbol of the algorithms is one IEEE
+                           round-to-nearest operation, in their order (roots, divisions and reciprocals
+                           by sequences that return the IEEE result: see ga_selftest_exact_forms).
+                           1: fast: approximate reciprocal and square root, one division per
+                           element (g*C/(|theta-theta^i|+C)); a few ulp off. Applies to GA_GA,
+                           GA_DANA_GA and GA_ADAM_GA (there also to Adam's own root and division);
+                           every other variant is always exact. On large vectors exact mode runs at
+                           the memory roofline too, so fast mode buys nothing there. */
     GA_OPT_STATS = 2,   /* 1: every arrival of GA_GA, GA_DANA_GA and GA_ADAM_GA also reduces the sum
                            and the maximum of the Gap over all parameters (the average Gap is what
                            Appendix "Gap and Delay" logs); read with ga_get_stats_window or
