@@ -389,6 +389,7 @@ void fill_window(ga_engine* e, ga::Window& w, const int* workers, const float* c
         w.saved[j] = e->row(i);
         w.vworker[j] = e->vrow(i);
         w.tau[j] = (float)tau;
+        w.inv_tau[j] = 1.0f / (float)tau;   // IEEE division on the host = the correctly rounded reciprocal
         w.bias1[j] = w.bias2[j] = 1.f;
         if (e->is_adam()) {   // Adam's bias corrections use the arrival index
             w.bias1[j] = ga_engine::inv_one_minus_pow(e->pow_b1, (double)e->gamma, k);
@@ -411,6 +412,7 @@ void fill_window(ga_engine* e, ga::Window& w, const int* workers, const float* c
         w.saved[j] = nullptr;
         w.vworker[j] = nullptr;
         w.tau[j] = 1.f;
+        w.inv_tau[j] = 1.f;
         w.bias1[j] = w.bias2[j] = 1.f;
         w.inv_bias[j] = 0.f;
         w.eta_eff[j] = 0.f;
@@ -1138,6 +1140,7 @@ extern "C" int64_t ga_selftest_exact_forms(int level, void* cuda_stream) {
     t::div_window<<<grid, block, 0, st>>>(-60, 127, -27, 65, -124, 100, 1u << 14, 3, bad);      // Adam's step
     for (float c : {0.1f, 0.01f, 1.0f, 0.001f, 0.5f}) t::div_const<<<grid, block, 0, st>>>(c, bad);
     t::gap_small_dist<<<grid, block, 0, st>>>(1u << 19, 4, bad);
+    t::div_by_delay<<<grid, block, 0, st>>>(16, 5, bad);                                          // Adam-SA's g / tau
     if (level >= 1)
         for (uint32_t slice = 0; slice < 64; ++slice) t::div_all_significands<<<1024, 128, 0, st>>>(slice << 17, bad);
     // the comparison itself is checked too: beyond 2^126 the short reciprocal is known to differ from
