@@ -182,6 +182,13 @@ def test_c2_heterogeneous_workers(P, variant):
     _sampled(P, "C2", variant, 16).close()
 
 
+@pytest.mark.parametrize("variant", ["DANA_GA", "ADAM_GA", "ADAM_SA", "SA_GRAD", "DANA_SA"])
+def test_c2_heterogeneous_workers_other_masters(P, variant):
+    """6,000 arrivals with widely spread delays (32 workers of log-normal speed) on the ResNet-20
+    shape -- short enough for the two-parameters-per-thread layout -- for the appendix's masters."""
+    _sampled(P, "C2", variant, 16, n_arrivals=6000).close()
+
+
 def test_c3_window_invariance(P):
     """ResNet-50 shape: K = 1, 4, 16 all match the oracle and each other, bit for bit."""
     import torch
