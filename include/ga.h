@@ -272,12 +272,16 @@ int64_t ga_selftest_exact_forms(int level, void* cuda_stream);
 /* Self-test of the bounded waits. The layer-wise kernels (GA_GA_LAYER) order consecutive arrivals by
  * waiting, layer by layer, for a counter that the previous arrival advances; like the bulk-copy waits
  * of ga_pull these waits have an iteration limit, after which the block raises the engine's error
- * flag and returns, and the engine reports GA_ERR_CUDA from its next synchronising call. This call
- * launches one block that waits for a counter nothing advances and checks that the wait runs out
- * (after about a second), that the flag is raised and that the kernel returns, leaving the
- * context usable. Returns GA_OK, GA_ERR_STATE if the wait did not behave so, or another negative
- * GA_ERR_* code. Allocates a few words for the duration of the call; synchronises cuda_stream. */
-int ga_selftest_bounded_wait(void* cuda_stream);
+ * flag and returns, and the engine reports GA_ERR_CUDA from its next synchronising call, for good.
+ * This call launches one block that waits for a counter nothing advances and checks that the wait
+ * runs out (after about a second), that the flag is raised and that the kernel returns, leaving the
+ * context usable. With engine == NULL it uses a flag of its own on cuda_stream. With an engine it
+ * raises THAT engine's flag (on the engine's stream; cuda_stream is ignored), which shows the whole
+ * reporting path: the call itself returns GA_OK, and every later synchronising call on the engine
+ * (ga_get, ga_get_stats, ...) returns GA_ERR_CUDA -- the engine is spent, as after a real lost wait.
+ * Returns GA_OK, GA_ERR_STATE if the wait did not behave so, or another negative GA_ERR_* code.
+ * Allocates a few words for the duration of the call; synchronises the stream. */
+int ga_selftest_bounded_wait(ga_engine* engine, void* cuda_stream);
 
 /* Gap statistics without any allocation. (The paper has no counterpart of this call; it exists
  * for deployment reasons only.) Computes the sum and the maximum over all parameters of the

@@ -60,7 +60,7 @@ _SIGNATURES = {
     "ga_gap_stats_noalloc": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_size_t, _c.c_float, _c.c_float,
                                         _c.c_int64, _c.c_void_p, _c.c_void_p]),
     "ga_selftest_exact_forms": (_c.c_int64, [_c.c_int, _c.c_void_p]),
-    "ga_selftest_bounded_wait": (_c.c_int, [_c.c_void_p]),
+    "ga_selftest_bounded_wait": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
     "ga_last_error": (_c.c_char_p, []),
 }
 

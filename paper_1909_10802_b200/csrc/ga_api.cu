@@ -1156,18 +1156,20 @@ extern "C" int64_t ga_selftest_exact_forms(int level, void* cuda_stream) {
 }
 
 // A wait inside the layer-wise kernels that nothing satisfies: it has to give up and say so.
-extern "C" int ga_selftest_bounded_wait(void* cuda_stream) {
-    cudaStream_t st = (cudaStream_t)cuda_stream;
+extern "C" int ga_selftest_bounded_wait(ga_engine* engine, void* cuda_stream) {
+    if (engine && engine->cuda_failed) return fail(GA_ERR_CUDA, "engine is unusable after an earlier CUDA error");
+    cudaStream_t st = engine ? engine->stream : (cudaStream_t)cuda_stream;
     unsigned int* epoch = nullptr;   // epoch word, then the abort word
     int* gave_up = nullptr;
-    int* flag = nullptr;   // mapped host memory, like an engine's error flag
+    int* own_flag = nullptr;         // mapped host memory, like an engine's error flag
     int rc = GA_OK;
     if (cudaMalloc(&epoch, 2 * sizeof *epoch) != cudaSuccess || cudaMalloc(&gave_up, sizeof *gave_up) != cudaSuccess ||
-        cudaHostAlloc(&flag, sizeof *flag, cudaHostAllocMapped) != cudaSuccess) {
+        (!engine && cudaHostAlloc(&own_flag, sizeof *own_flag, cudaHostAllocMapped) != cudaSuccess)) {
         cudaGetLastError();
         rc = fail(GA_ERR_OOM, "cannot allocate the probe's words");
     } else {
-        *flag = 0;
+        int* flag = engine ? engine->pull_err : own_flag;   // an engine's own flag: its next synchronising call reports it
+        if (!engine) *flag = 0;
         int host_gave_up = -1;
         cudaError_t err = cudaMemsetAsync(epoch, 0, 2 * sizeof *epoch, st);
         if (err == cudaSuccess) err = cudaMemsetAsync(gave_up, 0xff, sizeof *gave_up, st);
@@ -1183,7 +1185,7 @@ extern "C" int ga_selftest_bounded_wait(void* cuda_stream) {
     }
     cudaFree(epoch);
     cudaFree(gave_up);
-    if (flag) cudaFreeHost(flag);
+    if (own_flag) cudaFreeHost(own_flag);
     return rc;
 }
 

@@ -438,13 +438,24 @@ def test_a_wait_that_nothing_satisfies_gives_up_and_reports(P):
     import time
     import torch
     t0 = time.time()
-    assert P.lib().ga_selftest_bounded_wait(None) == P.GA_OK, P.last_error()
+    assert P.lib().ga_selftest_bounded_wait(None, None) == P.GA_OK, P.last_error()
     assert time.time() - t0 < 30.0
     eng = P.Engine(1000, 2, 0.1, 0.9, 0.999, P.GA_GA_LAYER)
     eng.set_params(torch.zeros(1000, device="cuda"))
     assert eng.push_batch([0, 1], [torch.ones(1000, device="cuda")] * 2) == [1, 2]
     assert torch.isfinite(eng.get(P.GA_THETA)).all()
+    # the same through an engine's own flag: the host learns of the lost wait at the next
+    # synchronising call, and the engine stays failed (every later call says so) while others work on
+    assert P.lib().ga_selftest_bounded_wait(eng._h, None) == P.GA_OK, P.last_error()
+    out = torch.empty(1000, device="cuda")
+    assert P.lib().ga_get(eng._h, P.GA_THETA, out.data_ptr()) == P.GA_ERR_CUDA and "waiting" in P.last_error()
+    assert P.lib().ga_push(eng._h, 0, out.data_ptr()) == P.GA_ERR_CUDA
     eng.close()
+    other = P.Engine(1000, 2, 0.1, 0.9, 0.999, P.GA_GA)
+    other.set_params(torch.zeros(1000, device="cuda"))
+    assert other.push_batch([0], [torch.ones(1000, device="cuda")]) == [1]
+    assert torch.isfinite(other.get(P.GA_THETA)).all()
+    other.close()
 
 
 # ----------------------------------------------------------------------------- caller-owned memory
