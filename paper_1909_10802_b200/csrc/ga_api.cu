@@ -208,6 +208,23 @@ int grid_1d(long long n, int threads, int cap) {
 
 // ----------------------------------------------------------------------------- launch
 
+// A launch that may be scheduled while the one before it on the stream is still draining (programmatic
+// dependent launch). The window kernel then waits for that launch to complete before it touches
+// memory; the layer kernels order themselves through the layers' epoch counters instead.
+template <typename... Params, typename... Args>
+cudaError_t launch_chained(void (*kernel)(Params...), long long grid, int block, cudaStream_t st, bool chained, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
+
 // stats_mode (STATS instantiations): 1 = the arrivals' pairs overwrite their log slots, 2 = they are
 // merged into them (a later chunk of the same arrivals on the host-buffer path)
 template <int FAMILY, int PENALTY, bool EXACT, int C_ORDER, bool STATS>
@@ -222,10 +239,12 @@ void launch_window_t(ga_engine* e, const ga::Window& w, long long vec_begin, lon
     if (STATS && blocks > e->stats_blocks) blocks = e->stats_blocks;
     // a single arrival has nothing to prefetch across: the one-arrival instantiation is leaner.
     constexpr int ST = GA_WINDOW_STAGES;
-#define GA_LAUNCH_V(BATCH, STAGES_, WD_, VEC_)                                                                   \
-    ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, BATCH, STAGES_, WD_, VEC_>                       \
-        <<<(unsigned)blocks, ga::kThreads, 0, st>>>(e->theta, e->vel, e->mom, e->sec, w, e->hyper(), first, last, \
-                                                    e->d, e->partials)
+    // launched so that it may be scheduled under the tail of the launch before it (the kernel waits for
+    // that launch to complete before its first access to global memory)
+#define GA_LAUNCH_V(BATCH, STAGES_, WD_, VEC_)                                                                       \
+    launch_chained(ga::ga_window_kernel<FAMILY, PENALTY, EXACT, C_ORDER, STATS, BATCH, STAGES_, WD_, VEC_>,           \
+                   (long long)blocks, ga::kThreads, st, true, e->theta, e->vel, e->mom, e->sec, w, e->hyper(), first, \
+                   last, e->d, e->partials)
 #define GA_LAUNCH(BATCH, STAGES_, WD_) \
     do { if (narrow) GA_LAUNCH_V(BATCH, STAGES_, WD_, 2); else GA_LAUNCH_V(BATCH, STAGES_, WD_, 4); } while (0)
     const bool wd = e->weight_decay != 0.f || e->nesterov;   // the instantiations with the extras
@@ -330,22 +349,6 @@ int build_layers(ga_engine* e, const int64_t* offsets, int n) {
     e->layer_off.assign(offsets, offsets + n + 1);
     e->n_tiles = (int)nt;
     return GA_OK;
-}
-
-// A launch that may begin while the one before it on the stream is still draining (programmatic
-// dependent launch); the kernels order themselves through the layers' epoch counters.
-template <typename... Params, typename... Args>
-cudaError_t launch_chained(void (*kernel)(Params...), int grid, int block, cudaStream_t st, bool chained, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3((unsigned)block);
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = chained ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
 }
 
 // Arrivals w.K of a window with the layer-wise Gap, one launch each, chained. The Gap of the

@@ -593,3 +593,34 @@ def test_host_buffer_path_on_a_short_vector(P, variant):
     for (s, m), (os_, om) in zip(eng.get_stats_window(), want):
         assert abs(s - os_) <= 1e-9 * os_ and m == om
     eng.close()
+
+
+@pytest.mark.parametrize("variant,d", [("GA", 272_474), ("GA", 3_000_001), ("DANA_GA", 272_474), ("ADAM_GA", 50_003),
+                                       ("SA", 272_474)])
+def test_calls_back_to_back_without_a_host_wait(P, variant, d):
+    """Window launches are made so that the next one may be scheduled under the tail of the one before
+    it (the kernel then waits for that launch to complete before it reads anything). Sixty calls of
+    one to eight arrivals on fixed gradients, nothing between them on the stream and no host wait:
+    the state and every saved copy equal the oracle's bit for bit."""
+    import torch
+    n = 8
+    rng = np.random.default_rng(d % 1000 + len(variant))
+    th0 = rng.normal(size=d).astype(np.float32)
+    pool = [(0.1 * rng.normal(size=d)).astype(np.float32) for _ in range(n)]
+    dev = [torch.from_numpy(g).cuda() for g in pool]
+    lr = 0.01 if variant.startswith("ADAM") else 0.1
+    o = oracle.Oracle(d, n, lr, 0.9, 0.999, oracle.VARIANTS[variant])
+    o.set_params(th0)
+    eng = P.Engine(d, n, lr, 0.9, 0.999, P.VARIANTS[variant])
+    eng.set_params(torch.from_numpy(th0).cuda())
+    calls = [[int(w) for w in rng.permutation(n)[: 1 + c % 8]] for c in range(60)]
+    got = [eng.push_batch(c, [dev[w] for w in c]) for c in calls]           # enqueued in one go
+    want = [o.push_batch(c, [pool[w] for w in c]) for c in calls]
+    assert got == want
+    for which, ow in ((P.GA_THETA, o.THETA), (P.GA_V, o.V), (P.GA_M, o.M)):
+        if which == P.GA_M and variant == "SA":
+            continue
+        assert np.array_equal(_np(eng.get(which)), o.get(ow).astype(np.float32)), (variant, which)
+    for w in range(n):
+        assert np.array_equal(_np(eng.saved(w)), o.saved(w).astype(np.float32)), w
+    eng.close()
