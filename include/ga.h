@@ -3,7 +3,7 @@
  * The library plays the master of asynchronous SGD with a parameter server
  * (arXiv 1909.10802, Section 4): it owns the master parameters theta, the momentum (update
  * vector) v, the running second moment m from which the coefficient C is derived, and one
- * saved copy of the parameters per worker (theta^i, "the parameters last sent to worker i").
+ * saved copy of the parameters per worker (theta^i: what was last sent to worker i).
  * Each arriving gradient is applied by one fused CUDA kernel; several consecutive arrivals
  * can be applied by a single launch that keeps theta, v and m in registers.
  *
