@@ -26,8 +26,13 @@ class Run:
                              workspace=workspace)    # workspace: a CUDA tensor that holds the engine's state
         self.engine.set_option(GA_OPT_WINDOW, window)
         if variant == "GA_LAYER":          # the workload's tensors are the layers
-            assert shard is None, "a layer's norm needs the whole layer on one rank"
-            self.engine.set_layers(wl.seg_off)
+            # a layer's norm needs the whole layer on one rank: a shard must begin and end on layer
+            # boundaries (shard.layer_shard_range), and holds the layers in between
+            off = [int(x) for x in wl.seg_off]
+            if self.j0 not in off or self.j0 + self.n not in off:
+                raise ValueError("a shard of the layer-wise Gap must consist of whole layers")
+            l0, l1 = off.index(self.j0), off.index(self.j0 + self.n)
+            self.engine.set_layers([x - self.j0 for x in off[l0:l1 + 1]])
         for key, value in (options or {}).items():
             self.engine.set_option(key, value)
         theta0 = torch.empty(self.n, dtype=torch.float32, device=torch_device)

@@ -14,8 +14,13 @@ def run_oracle(wl, variant, n_arrivals=None, idx=None, precision=32, c_order=0, 
                       oracle.VARIANTS[variant],
                       precision=precision, c_order=c_order)
     if variant == "GA_LAYER":
-        assert idx is None, "layer norms need whole layers"
-        o.set_layers(wl.seg_off)
+        if idx is None:
+            o.set_layers(wl.seg_off)
+        else:                        # a contiguous range made of whole layers: those layers alone
+            off = [int(x) for x in wl.seg_off]
+            j0, j1 = int(idx[0]), int(idx[-1]) + 1
+            assert len(idx) == j1 - j0 and j0 in off and j1 in off, "layer norms need whole layers"
+            o.set_layers([x - j0 for x in off[off.index(j0):off.index(j1) + 1]])
     o.set_params(wl.theta0(idx))
     sched = (schedule if schedule is not None else wl.schedule())
     sched = sched[:n_arrivals if n_arrivals is not None else len(sched)]

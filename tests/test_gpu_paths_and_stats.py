@@ -624,3 +624,36 @@ def test_calls_back_to_back_without_a_host_wait(P, variant, d):
     for w in range(n):
         assert np.array_equal(_np(eng.saved(w)), o.saved(w).astype(np.float32)), w
     eng.close()
+
+
+@pytest.mark.parametrize("config,world,n_arrivals", [("mini", 2, None), ("C1", 3, 120)])
+def test_layer_wise_gap_on_shards_of_whole_layers(P, config, world, n_arrivals):
+    """The layer-wise Gap (Section 5.3) with the vector split over ranks at layer boundaries: each
+    engine holds whole layers and needs nothing from the others. One shard after the other on one
+    GPU; parameters, momentum, a saved copy, the per-layer Gaps and second moments, put together,
+    equal the oracle's run over the whole vector bit for bit."""
+    from paper_1909_10802_b200.runner import Run
+    from paper_1909_10802_b200.shard import layer_shard_range
+    wl = W.config(config)
+    o, odelays, _ = run_oracle(wl, "GA_LAYER", n_arrivals=n_arrivals)
+    ogap, om = o.layer_state()
+    theta, vel, saved, gaps, ms = [], [], [], [], []
+    for rank in range(world):
+        l0, l1, j0, n = layer_shard_range(wl.seg_off, rank, world)
+        part = Run(wl, "GA_LAYER", 16, shard=(j0, n))
+        assert part.engine.n_layers == l1 - l0
+        assert part.run(n_arrivals) == odelays
+        theta.append(_np(part.engine.get(P.GA_THETA)))
+        vel.append(_np(part.engine.get(P.GA_V)))
+        saved.append(_np(part.engine.saved(1)))
+        g, m = part.engine.get_layer_state()
+        gaps.append(g)
+        ms.append(m)
+        part.close()
+    assert np.array_equal(np.concatenate(theta), o.get(o.THETA).astype(np.float32))
+    assert np.array_equal(np.concatenate(vel), o.get(o.V).astype(np.float32))
+    assert np.array_equal(np.concatenate(saved), o.saved(1).astype(np.float32))
+    assert np.array_equal(np.concatenate(gaps), ogap.astype(np.float32))
+    assert np.array_equal(np.concatenate(ms), om.astype(np.float32))
+    with pytest.raises(ValueError):           # a range that cuts a layer is refused
+        Run(wl, "GA_LAYER", 16, shard=(0, int(wl.seg_off[1]) + 1))

@@ -74,3 +74,33 @@ def test_shards_tile_the_vector(d, world):
         assert j0 == pos and n >= 0 and (j0 % 32 == 0 or n == 0)
         pos += n
     assert pos == d
+
+
+@pytest.mark.parametrize("config,world", [("C1", 2), ("C1", 3), ("C3", 8), ("C3", 5), ("C4", 4), ("C5", 2), ("mini", 2)])
+def test_layer_shards_hold_whole_layers_and_tile_the_vector(config, world):
+    """Ranks of the layer-wise Gap own whole layers: consecutive, non-empty, covering every layer once;
+    where no layer dominates (the ResNet shapes) no rank is more than one layer away from an equal share."""
+    import workloads as W
+    from paper_1909_10802_b200.shard import layer_shard_range
+    off = [int(x) for x in W.config(config).seg_off]
+    d, biggest = off[-1], max(b - a for a, b in zip(off, off[1:]))
+    pos_l, pos_j = 0, 0
+    for r in range(world):
+        l0, l1, j0, n = layer_shard_range(off, r, world)
+        assert l0 == pos_l and l1 > l0 and j0 == pos_j == off[l0] and n == off[l1] - off[l0]
+        if config in ("C1", "C3", "C4"):
+            assert abs(n - d / world) <= biggest
+        pos_l, pos_j = l1, j0 + n
+    assert pos_l == len(off) - 1 and pos_j == d
+
+
+def test_layer_shards_refuse_what_cannot_be_split():
+    from paper_1909_10802_b200.shard import layer_shard_range
+    with pytest.raises(ValueError):
+        layer_shard_range([0, 10, 20], 0, 3)          # more ranks than layers
+    with pytest.raises(ValueError):
+        layer_shard_range([0, 10, 10], 0, 1)          # an empty layer
+    with pytest.raises(ValueError):
+        layer_shard_range([0, 10, 20], 2, 2)
+    assert layer_shard_range([0, 10, 20], 1, 2) == (1, 2, 10, 10)
+    assert layer_shard_range([0, 1, 2, 1000], 0, 2) == (0, 2, 0, 2)      # a dominant layer stays whole

@@ -62,3 +62,35 @@ def test_two_ranks_equal_one(tmp_path):
     for r in range(world):
         got_sum, got_max = np.load(tmp_path / f"stats_{r}.npy")
         assert abs(got_sum - want_sum) <= 1e-12 * want_sum and got_max == want_max
+
+
+def _layer_rank(rank, world, port, out_dir):
+    import torch.distributed as dist
+    from paper_1909_10802_b200.shard import assert_same_schedule, layer_shard_range
+    from tests.oracle_run import run_oracle
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = W.config("mini")
+    assert_same_schedule(wl.schedule(), dist)
+    l0, l1, j0, n = layer_shard_range(wl.seg_off, rank, world)
+    o, delays, _ = run_oracle(wl, "GA_LAYER", idx=np.arange(j0, j0 + n, dtype=np.int64))
+    gaps, m_layers = o.layer_state()
+    np.save(os.path.join(out_dir, f"ltheta_{rank}.npy"), o.get(o.THETA))
+    np.save(os.path.join(out_dir, f"lgap_{rank}.npy"), np.asarray(gaps))
+    np.save(os.path.join(out_dir, f"lm_{rank}.npy"), np.asarray(m_layers))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_layer_wise_gap_on_ranks_that_hold_whole_layers(tmp_path):
+    """Section 5.3's layer-wise Gap on two ranks: each holds whole layers, nothing is exchanged, and
+    parameters, per-layer Gaps and per-layer second moments together are the single-rank run's."""
+    from tests.oracle_run import run_oracle
+    world = 2
+    mp.spawn(_layer_rank, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    wl = W.config("mini")
+    full, _, _ = run_oracle(wl, "GA_LAYER")
+    gaps, m_layers = full.layer_state()
+    cat = lambda name: np.concatenate([np.load(tmp_path / f"{name}_{r}.npy") for r in range(world)])
+    assert np.array_equal(cat("ltheta"), full.get(full.THETA))
+    assert np.array_equal(cat("lgap"), np.asarray(gaps)) and np.array_equal(cat("lm"), np.asarray(m_layers))
