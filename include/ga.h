@@ -63,8 +63,8 @@ enum {
      * update vector. Norms are accumulated in fp64 and rounded to fp32 once. A layer's norm must be
      * known before the layer is updated, so arrivals are not fused in time: each is one launch over
      * the vector, which inside a ga_push_batch call also measures the next arrival's distance (one
-     * extra distance pass per call), and consecutive launches overlap. ga_push_batch_host is not
-     * available for this variant. */
+     * extra distance pass per call), and consecutive launches overlap. ga_push_batch_host stages
+     * whole gradients for this variant (see there). */
     GA_GA_LAYER = 10
 };
 
@@ -203,7 +203,10 @@ int ga_push_batch(ga_engine* e, const int* schedule_host, const float* const* gr
  * schedule[j] after its arrival (n_params floats each). The parameter range is processed in
  * chunks so that host-to-device copies, the update kernel and device-to-host copies overlap,
  * across the windows of the call as well as within them. Synchronous: returns when all results
- * are in host memory. Allocates its staging buffers (2 x 16 x 16 MiB) on first use. */
+ * are in host memory. Allocates its staging buffers (2 x 16 x 16 MiB) on first use.
+ * GA_GA_LAYER needs a whole gradient before a layer's norm is known: there the call stages whole
+ * vectors, one arrival at a time (two staging buffers of n_params floats), the copy-in of the next
+ * arrival and the copy-out of the previous one running beside the launches of the current. */
 int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* const* grads_host,
                        int K, int64_t* delays_out_host, float* const* sent_out_host);
 

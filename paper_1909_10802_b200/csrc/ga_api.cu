@@ -40,6 +40,7 @@ constexpr long long kRowAlign = 32;            // floats: rows start on 128-byte
 constexpr long long kHostChunk = GA_HOST_CHUNK_FLOATS;   // floats per chunk of the host-buffer path
 constexpr int kHostStages = GA_HOST_STAGES;              // staging buffers the copies-in rotate through
 constexpr int kHostD2hRing = 4;                // chunks the kernels may run ahead of the copies out
+constexpr int kLayerHostGroup = 1;             // whole gradient vectors per staging buffer (layer-wise Gap)
 constexpr uint32_t kStateMagic = 0x47415331;   // "GAS1"
 constexpr int kStatsLog = GA_STATS_LOG;        // arrivals whose Gap statistics are kept
 
@@ -448,10 +449,13 @@ int validate_batch(ga_engine* e, const int* schedule, const void* const* bufs, i
 
 int ensure_host_path(ga_engine* e) {
     if (e->stage[0]) return GA_OK;
-    const long long chunk = e->stride < kHostChunk ? e->stride : kHostChunk;
+    // parameter-wise masters stage a chunk of every gradient of a window; the layer-wise Gap needs
+    // whole vectors before a layer's norm is known, so it stages a few whole gradients instead
+    const long long chunk = e->is_layer() ? e->stride : (e->stride < kHostChunk ? e->stride : kHostChunk);
+    const int per_stage = e->is_layer() ? kLayerHostGroup : ga::kMaxWindow;
     e->stage_elems = chunk;
     for (int s = 0; s < kHostStages; ++s) {
-        if (cudaMalloc(&e->stage[s], sizeof(float) * (size_t)chunk * ga::kMaxWindow) != cudaSuccess) {
+        if (cudaMalloc(&e->stage[s], sizeof(float) * (size_t)chunk * per_stage) != cudaSuccess) {
             cudaGetLastError();
             return fail(GA_ERR_OOM, "cannot allocate staging buffers for the host-buffer path");
         }
@@ -799,11 +803,55 @@ int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* cons
     if (sent_out_host)
         for (int j = 0; j < K; ++j)
             if (!sent_out_host[j]) return fail(GA_ERR_ARG, "sent_out_host[%d] is NULL", j);
-    if (e->is_layer()) return fail(GA_ERR_STATE, "the layer-wise Gap needs whole vectors on the device: use ga_push_batch");
     DeviceGuard guard(e->device);
     if (int rc = ensure_host_path(e)) return rc;
     int launches = 0;
     if (K > 0) e->stats_total = 0;
+    if (e->is_layer()) {
+        // Whole gradients, kLayerHostGroup arrivals at a time: copies-in of group g+1 and copies-out
+        // of group g-1 run beside the launches of group g (one distance pass + one launch per
+        // arrival). A group ends where a worker would repeat, so every sent copy is read out before
+        // it is written again. Small groups keep the call's first copy-in and last copy-out, which
+        // nothing overlaps, short.
+        GA_CUDA(e, cudaEventRecord(e->ev_prev, e->stream));
+        GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_prev, 0));
+        GA_CUDA(e, cudaStreamWaitEvent(e->s_d2h, e->ev_prev, 0));
+        const int group = e->window < kLayerHostGroup ? e->window : kLayerHostGroup;
+        const size_t vec_bytes = sizeof(float) * (size_t)e->d;
+        long long g = 0;
+        for (int pos = 0; pos < K; ++g) {
+            const int n = next_window(schedule_host, pos, K, group);
+            const int s = (int)(g % kHostStages);
+            if (g >= kHostStages) GA_CUDA(e, cudaStreamWaitEvent(e->s_h2d, e->ev_kernel[s], 0));
+            const float* staged[ga::kMaxWindow] = {};
+            for (int j = 0; j < n; ++j) {
+                float* dst = e->stage[s] + (size_t)j * e->stride;
+                GA_CUDA(e, cudaMemcpyAsync(dst, grads_host[pos + j], vec_bytes, cudaMemcpyHostToDevice, e->s_h2d));
+                staged[j] = dst;
+            }
+            GA_CUDA(e, cudaEventRecord(e->ev_h2d[s], e->s_h2d));
+            GA_CUDA(e, cudaStreamWaitEvent(e->stream, e->ev_h2d[s], 0));
+            // the copies out of the group before this one read saved rows that this group may rewrite
+            if (sent_out_host && g >= 1) GA_CUDA(e, cudaStreamWaitEvent(e->stream, e->ev_d2h[(g - 1) % kHostD2hRing], 0));
+            ga::Window w;
+            fill_window(e, w, schedule_host + pos, staged, n, true, delays_out_host ? delays_out_host + pos : nullptr);
+            if (int rc = launch_layer_arrivals(e, w, false, nullptr, 0.f)) return rc;
+            launches += n + 1;
+            GA_CUDA(e, cudaEventRecord(e->ev_kernel[s], e->stream));
+            if (sent_out_host) {
+                GA_CUDA(e, cudaStreamWaitEvent(e->s_d2h, e->ev_kernel[s], 0));
+                for (int j = 0; j < n; ++j)
+                    GA_CUDA(e, cudaMemcpyAsync(sent_out_host[pos + j], e->row(schedule_host[pos + j]), vec_bytes,
+                                               cudaMemcpyDeviceToHost, e->s_d2h));
+                GA_CUDA(e, cudaEventRecord(e->ev_d2h[g % kHostD2hRing], e->s_d2h));
+            }
+            pos += n;
+        }
+        GA_CUDA(e, cudaStreamSynchronize(e->s_h2d));
+        GA_CUDA(e, cudaStreamSynchronize(e->s_d2h));
+        if (int rc = sync_and_check(e)) return rc;
+        return launches;
+    }
     const long long chunk = e->stage_elems;
     const long long n_chunks = (e->stride + chunk - 1) / chunk;
     // How far the update kernels may run ahead of the copies back to the host. The kernel of

@@ -657,3 +657,44 @@ def test_layer_wise_gap_on_shards_of_whole_layers(P, config, world, n_arrivals):
     assert np.array_equal(np.concatenate(ms), om.astype(np.float32))
     with pytest.raises(ValueError):           # a range that cuts a layer is refused
         Run(wl, "GA_LAYER", 16, shard=(0, int(wl.seg_off[1]) + 1))
+
+
+def test_host_buffer_path_with_the_layer_wise_gap(P):
+    """ga_push_batch_host for the layer-wise Gap (Section 5.3): whole gradients are staged a few
+    arrivals at a time. Eleven arrivals with workers that repeat (next to one another and further
+    apart), a ragged vector in five layers: the parameters sent after every arrival, the state and
+    the per-layer Gaps and second moments equal the oracle's, and so does a second call."""
+    import torch
+    d, n = 20_011, 4
+    layers = [0, 4096, 4100, 12_000, 12_001, d]
+    rng = np.random.default_rng(21)
+    th0 = rng.normal(size=d).astype(np.float32)
+    sched = [1, 0, 2, 3, 3, 0, 1, 2, 0, 0, 3]
+    grads = [(0.1 * rng.normal(size=d)).astype(np.float32) for _ in sched]
+    o = oracle.Oracle(d, n, 0.1, 0.9, 0.999, oracle.GA_LAYER)
+    o.set_layers(layers)
+    o.set_params(th0)
+    eng = P.Engine(d, n, 0.1, 0.9, 0.999, P.GA_GA_LAYER)
+    eng.set_layers(layers)
+    eng.set_params(torch.from_numpy(th0).cuda())
+    for call in range(2):
+        want_sent, want_delays = [], []
+        for i, g in zip(sched, grads):
+            want_delays.append(o.push(i, g))
+            o.pull(i)
+            want_sent.append(o.saved(i).astype(np.float32))
+        outs = [torch.empty(d, dtype=torch.float32).pin_memory() for _ in sched]
+        got_delays, launches = eng.push_batch_host(sched, [torch.from_numpy(g).pin_memory() for g in grads], outs)
+        assert got_delays == want_delays and launches > len(sched)      # one launch per arrival + distance passes
+        for j, (got, want) in enumerate(zip(outs, want_sent)):
+            assert np.array_equal(got.numpy(), want), (call, j)
+        assert np.array_equal(_np(eng.get(P.GA_THETA)), o.get(o.THETA).astype(np.float32))
+        assert np.array_equal(_np(eng.get(P.GA_V)), o.get(o.V).astype(np.float32))
+        ogap, om = o.layer_state()
+        gap, m = eng.get_layer_state()
+        assert np.array_equal(gap, ogap.astype(np.float32)) and np.array_equal(m, om.astype(np.float32))
+    # and the device path carries on from there
+    dev = [torch.from_numpy(g).cuda() for g in grads[:3]]
+    assert eng.push_batch([2, 2, 1], dev) == o.push_batch([2, 2, 1], grads[:3])
+    assert np.array_equal(_np(eng.get(P.GA_THETA)), o.get(o.THETA).astype(np.float32))
+    eng.close()
