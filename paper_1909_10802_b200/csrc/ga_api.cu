@@ -83,6 +83,7 @@ struct ga_engine {
     ga::StatsPartial* partials = nullptr;
     double* stats_dev = nullptr;   // ring of kStatsLog x {sum, max}: one pair per arrival
     int stats_blocks = 0;
+    int sms = 148;                 // multiprocessors of the engine's device
     int small_range_vectors = 0;   // ranges of fewer 16-byte vectors than this run with two parameters per thread
     int64_t stats_total = 0;       // arrivals logged since the current call began (slot = index % kStatsLog)
     // pull kernel error flag: one int of pinned, device-mapped host memory
@@ -540,8 +541,8 @@ ga_engine* create_engine(size_t n_params, int n_workers, float lr, float momentu
         return nullptr;
     }
     cudaDeviceProp prop;
-    int sms = 148;
-    if (cudaGetDeviceProperties(&prop, e->device) == cudaSuccess) sms = prop.multiProcessorCount;
+    if (cudaGetDeviceProperties(&prop, e->device) == cudaSuccess) e->sms = prop.multiProcessorCount;
+    const int sms = e->sms;
     e->stats_blocks = sms * 8 < kMaxStatsBlocks ? sms * 8 : kMaxStatsBlocks;
     e->small_range_vectors = sms * 9 * ga::kThreads;   // one full set of resident blocks at four parameters per thread
     const size_t row_bytes = sizeof(float) * (size_t)e->stride;
@@ -696,7 +697,7 @@ int ga_set_params(ga_engine* e, const float* theta0_dev) {
     if (int rc = check_engine(e)) return rc;
     if (int rc = check_dev_ptr(theta0_dev, "theta0_dev")) return rc;
     DeviceGuard guard(e->device);
-    ga::ga_set_params_kernel<<<grid_1d(e->stride, 256, 148 * 8), 256, 0, e->stream>>>(
+    ga::ga_set_params_kernel<<<grid_1d(e->stride, 256, e->sms * 8), 256, 0, e->stream>>>(
         theta0_dev, e->theta, e->vel, e->mom, e->saved, e->vworker, e->n_workers, e->d, e->stride);
     GA_CUDA(e, cudaGetLastError());
     if (e->sec) GA_CUDA(e, cudaMemsetAsync(e->sec, 0, sizeof(float) * (size_t)e->stride, e->stream));
@@ -712,7 +713,7 @@ const float* ga_pull(ga_engine* e, int worker) {
     if (check_engine(e) || check_worker(e, worker)) return nullptr;
     DeviceGuard guard(e->device);
     if (e->is_dana()) {   // the worker is sent the look-ahead estimate, not theta
-        ga::ga_pull_estimate_kernel<<<grid_1d(e->stride, 256, 148 * 8), 256, 0, e->stream>>>(
+        ga::ga_pull_estimate_kernel<<<grid_1d(e->stride, 256, e->sms * 8), 256, 0, e->stream>>>(
             e->theta, e->vel, e->hyper().eta_gamma, e->stride, e->row(worker));
         cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) { cuda_fail(e, err, "ga_pull launch"); return nullptr; }
@@ -721,7 +722,7 @@ const float* ga_pull(ga_engine* e, int worker) {
     }
     const long long bytes = e->stride * (long long)sizeof(float);
     const long long chunks = (bytes + ga::kPullChunk - 1) / ga::kPullChunk;
-    const long long max_grid = (long long)(e->stats_blocks / 8) * ga::kPullBlocksPerSm;   // SMs x blocks per SM
+    const long long max_grid = (long long)e->sms * ga::kPullBlocksPerSm;
     const int grid = (int)(chunks < max_grid ? chunks : max_grid);
     ga::ga_pull_bulk_kernel<<<grid, 32, ga::kPullStages * ga::kPullChunk, e->stream>>>(
         e->theta, e->row(worker), bytes, e->pull_err);
@@ -920,7 +921,7 @@ int ga_get(ga_engine* e, int which, float* out_dev) {
     } else if (which == GA_C && e->is_layer()) {
         return fail(GA_ERR_STATE, "the layer-wise variant has one C per layer: see ga_get_layer_state");
     } else if (which == GA_C) {
-        ga::ga_coeff_kernel<<<grid_1d(e->d, 256, 148 * 8), 256, 0, e->stream>>>(e->mom, e->inv_bias(e->k_c),
+        ga::ga_coeff_kernel<<<grid_1d(e->d, 256, e->sms * 8), 256, 0, e->stream>>>(e->mom, e->inv_bias(e->k_c),
                                                                                e->hyper(), e->d, out_dev);
         GA_CUDA(e, cudaGetLastError());
     } else {
@@ -945,7 +946,7 @@ int ga_gap(ga_engine* e, int worker, float* gap_out_dev) {
     if (int rc = check_dev_ptr(gap_out_dev, "gap_out_dev")) return rc;
     if (e->is_layer()) return fail(GA_ERR_STATE, "the layer-wise variant has one Gap per layer: see ga_get_layer_state");
     DeviceGuard guard(e->device);
-    ga::ga_gap_kernel<<<grid_1d(e->d, 256, 148 * 8), 256, 0, e->stream>>>(
+    ga::ga_gap_kernel<<<grid_1d(e->d, 256, e->sms * 8), 256, 0, e->stream>>>(
         e->theta, e->row(worker), e->mom, e->inv_bias(e->k_c), e->hyper(), e->d, gap_out_dev);
     GA_CUDA(e, cudaGetLastError());
     return sync_and_check(e);
