@@ -693,8 +693,46 @@ def test_host_buffer_path_with_the_layer_wise_gap(P):
         ogap, om = o.layer_state()
         gap, m = eng.get_layer_state()
         assert np.array_equal(gap, ogap.astype(np.float32)) and np.array_equal(m, om.astype(np.float32))
-    # and the device path carries on from there
+    # without copies back to the host, and then the device path carries on from there
+    got_delays, _ = eng.push_batch_host([0, 0, 2], [torch.from_numpy(g).pin_memory() for g in grads[3:6]])
+    assert got_delays == o.push_batch([0, 0, 2], grads[3:6])
     dev = [torch.from_numpy(g).cuda() for g in grads[:3]]
     assert eng.push_batch([2, 2, 1], dev) == o.push_batch([2, 2, 1], grads[:3])
     assert np.array_equal(_np(eng.get(P.GA_THETA)), o.get(o.THETA).astype(np.float32))
+    assert np.array_equal(_np(eng.saved(0)), o.saved(0).astype(np.float32))
     eng.close()
+
+
+def test_engines_give_their_memory_back(P):
+    """Create, use (device path, host-buffer path with its staging buffers and streams, layer tables,
+    statistics) and destroy engines of every kind many times: the device's free memory afterwards is
+    what it was before."""
+    import torch
+    d, n = 300_001, 3
+    g = torch.ones(d, device="cuda")
+    gh = torch.ones(d).pin_memory()
+    out = torch.empty(d).pin_memory()
+
+    def cycle(variant):
+        eng = P.Engine(d, n, 0.01, 0.9, 0.999, P.VARIANTS[variant])
+        if variant == "GA_LAYER":
+            eng.set_layers([0, 1000, 200_000, d])
+        elif variant in GAP_VARIANTS:
+            eng.set_option(P.GA_OPT_STATS, 1)
+        eng.set_params(g)
+        eng.push_batch([0, 1], [g, g])
+        eng.push_batch_host([2, 0], [gh, gh], [out, out])
+        eng.pull(1)
+        eng.close()
+
+    kinds = ["GA", "SA", "DANA_GA", "ADAM_GA", "GA_LAYER"]
+    for v in kinds:
+        cycle(v)                              # first use: lazily created contexts, module loading
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(40):
+        for v in kinds:
+            cycle(v)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 >= free0 - (8 << 20), (free0, free1)      # nothing of the 200 engines (tens of MB each) is left
