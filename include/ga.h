@@ -139,7 +139,9 @@ ga_engine* ga_create_in(size_t n_params, int n_workers, float lr, float momentum
 /* Free everything the engine owns. NULL is accepted. Synchronises the bound stream first. */
 void ga_destroy(ga_engine* e);
 
-/* Enqueue all later work of this engine on cuda_stream (a cudaStream_t; NULL = default stream). */
+/* Enqueue all later work of this engine on cuda_stream (a cudaStream_t; NULL = default stream).
+ * The new stream is made to wait (by an event) for the work this engine has already enqueued on
+ * the stream it leaves, so a change of stream never reorders the engine's own launches. */
 int ga_set_stream(ga_engine* e, void* cuda_stream);
 
 /* Learning rate eta_k for the arrivals that follow (decay, warm-up: Appendix "Hyperparameters").

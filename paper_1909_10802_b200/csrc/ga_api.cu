@@ -652,7 +652,19 @@ void ga_destroy(ga_engine* e) {
 
 int ga_set_stream(ga_engine* e, void* cuda_stream) {
     if (int rc = check_engine(e)) return rc;
-    e->stream = (cudaStream_t)cuda_stream;
+    cudaStream_t next = (cudaStream_t)cuda_stream;
+    if (next != e->stream) {
+        // what the engine already enqueued on the old stream comes before anything it enqueues on
+        // the new one: every launch reads the state the launch before it wrote
+        DeviceGuard guard(e->device);
+        cudaEvent_t done = nullptr;
+        GA_CUDA(e, cudaEventCreateWithFlags(&done, cudaEventDisableTiming));
+        cudaError_t err = cudaEventRecord(done, e->stream);
+        if (err == cudaSuccess) err = cudaStreamWaitEvent(next, done, 0);
+        cudaEventDestroy(done);   // released once the record has completed
+        GA_CUDA(e, err);
+        e->stream = next;
+    }
     return GA_OK;
 }
 

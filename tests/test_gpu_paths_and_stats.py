@@ -736,3 +736,30 @@ def test_engines_give_their_memory_back(P):
     torch.cuda.synchronize()
     free1, _ = torch.cuda.mem_get_info()
     assert free1 >= free0 - (8 << 20), (free0, free1)      # nothing of the 200 engines (tens of MB each) is left
+
+
+@pytest.mark.parametrize("variant", ["GA", "GA_LAYER"])
+def test_a_change_of_stream_keeps_the_engines_launches_in_order(P, variant):
+    """ga_set_stream while work is still queued on the old stream: the new stream waits for it, so
+    windows enqueued on alternating streams, with no host wait in between, give the oracle's result."""
+    import torch
+    d, n = 6_000_011, 4
+    rng = np.random.default_rng(33)
+    th0 = rng.normal(size=d).astype(np.float32)
+    pool = [(0.1 * rng.normal(size=d)).astype(np.float32) for _ in range(n)]
+    dev = [torch.from_numpy(g).cuda() for g in pool]
+    o = oracle.Oracle(d, n, 0.1, 0.9, 0.999, oracle.VARIANTS[variant])
+    o.set_params(th0)
+    eng = P.Engine(d, n, 0.1, 0.9, 0.999, P.VARIANTS[variant])
+    eng.set_params(torch.from_numpy(th0).cuda())
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    calls = [[0, 1, 2, 3], [2, 0], [3, 1, 0], [1], [0, 2, 3, 1], [3, 0]]
+    for c, call in enumerate(calls):
+        eng.set_stream(streams[c % 2])
+        assert eng.push_batch(call, [dev[w] for w in call]) == o.push_batch(call, [pool[w] for w in call])
+    assert np.array_equal(_np(eng.get(P.GA_THETA)), o.get(o.THETA).astype(np.float32))
+    assert np.array_equal(_np(eng.get(P.GA_V)), o.get(o.V).astype(np.float32))
+    for w in range(n):
+        assert np.array_equal(_np(eng.saved(w)), o.saved(w).astype(np.float32))
+    eng.close()
