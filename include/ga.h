@@ -12,7 +12,11 @@
  *     n_params floats; pointers named *_host are HOST pointers. The library owns theta, v, m
  *     and the saved copies (allocated in ga_create, freed in ga_destroy); the caller owns
  *     gradient buffers and every output buffer it passes in, and must keep a gradient buffer
- *     unchanged until the work enqueued by the call that reads it has finished.
+ *     unchanged until the work enqueued by the call that reads it has finished. A *_dev pointer
+ *     that the CUDA runtime reports as ordinary host memory, or as memory of a device that the
+ *     engine's device cannot reach, is refused with GA_ERR_ARG before any kernel could touch it
+ *     (asked once per pointer; pinned and managed memory pass). The length of a caller's buffer
+ *     cannot be checked: a buffer shorter than n_params floats is the caller's error.
  *   - Work is enqueued on the stream bound with ga_set_stream (default: the legacy default
  *     stream) and the call returns after host bookkeeping; ga_get, ga_gap, ga_get_stats,
  *     ga_export_state and the *_host calls synchronise that stream before returning.

@@ -86,6 +86,8 @@ struct ga_engine {
     int sms = 148;                 // multiprocessors of the engine's device
     int small_range_vectors = 0;   // ranges of fewer 16-byte vectors than this run with two parameters per thread
     int64_t stats_total = 0;       // arrivals logged since the current call began (slot = index % kStatsLog)
+    const void* known_dev_ptrs[64] = {};   // caller's device pointers already looked up (check_dev_ptr)
+    unsigned known_dev_next = 0;
     // pull kernel error flag: one int of pinned, device-mapped host memory
     int* pull_err = nullptr;
     // beta^k, gamma^k, beta2^k carried from one arrival to the next (see inv_one_minus_pow)
@@ -185,6 +187,35 @@ int check_worker(ga_engine* e, int worker) {
 int check_dev_ptr(const void* p, const char* name) {
     if (!p) return fail(GA_ERR_ARG, "%s is NULL", name);
     if ((uintptr_t)p % 16) return fail(GA_ERR_ARG, "%s is not 16-byte aligned", name);
+    return GA_OK;
+}
+
+// The same for an engine's call, plus: is this memory a kernel of the engine's device can read? A
+// pointer to ordinary host memory handed over as a device pointer would fault the kernel that
+// dereferences it, so the runtime is asked once per pointer (callers reuse their gradient buffers:
+// the last 64 accepted pointers are remembered). Pinned or managed memory passes: the device can reach it.
+bool known_dev_ptr(const ga_engine* e, const void* p) {
+    for (const void* seen : e->known_dev_ptrs)
+        if (seen == p) return true;
+    return false;
+}
+
+int check_dev_ptr(ga_engine* e, const void* p, const char* name) {
+    if (int rc = check_dev_ptr(p, name)) return rc;
+    if (known_dev_ptr(e, p)) return GA_OK;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(GA_ERR_ARG, "%s is not memory the CUDA runtime knows", name);
+    }
+    if (attr.type == cudaMemoryTypeUnregistered)
+        return fail(GA_ERR_ARG, "%s points to ordinary host memory, not to device memory", name);
+    if (attr.type == cudaMemoryTypeDevice && attr.device != e->device) {
+        int reachable = 0;
+        cudaDeviceCanAccessPeer(&reachable, e->device, attr.device);
+        if (!reachable) return fail(GA_ERR_ARG, "%s lives on device %d, which device %d cannot reach", name, attr.device, e->device);
+    }
+    e->known_dev_ptrs[e->known_dev_next++ % (sizeof e->known_dev_ptrs / sizeof e->known_dev_ptrs[0])] = p;
     return GA_OK;
 }
 
@@ -443,7 +474,11 @@ int validate_batch(ga_engine* e, const int* schedule, const void* const* bufs, i
     for (int j = 0; j < K; ++j) {
         if (int rc = check_worker(e, schedule[j])) return rc;
         if (!bufs[j]) return fail(GA_ERR_ARG, "gradient %d is NULL", j);
-        if (device_ptrs && (uintptr_t)bufs[j] % 16) return fail(GA_ERR_ARG, "gradient %d is not 16-byte aligned", j);
+        if (device_ptrs && ((uintptr_t)bufs[j] % 16 || !known_dev_ptr(e, bufs[j]))) {   // not seen before: the full check
+            char name[32];
+            snprintf(name, sizeof name, "gradient %d", j);
+            if (int rc = check_dev_ptr(e, bufs[j], name)) return rc;
+        }
     }
     return GA_OK;
 }
@@ -707,7 +742,7 @@ int ga_get_layer_state(ga_engine* e, float* gaps_host, float* m_host) {
 
 int ga_set_params(ga_engine* e, const float* theta0_dev) {
     if (int rc = check_engine(e)) return rc;
-    if (int rc = check_dev_ptr(theta0_dev, "theta0_dev")) return rc;
+    if (int rc = check_dev_ptr(e, theta0_dev, "theta0_dev")) return rc;
     DeviceGuard guard(e->device);
     ga::ga_set_params_kernel<<<grid_1d(e->stride, 256, e->sms * 8), 256, 0, e->stream>>>(
         theta0_dev, e->theta, e->vel, e->mom, e->saved, e->vworker, e->n_workers, e->d, e->stride);
@@ -752,7 +787,7 @@ const float* ga_saved(ga_engine* e, int worker) {
 int64_t ga_push(ga_engine* e, int worker, const float* grad_dev) {
     if (int rc = check_engine(e)) return rc;
     if (int rc = check_worker(e, worker)) return rc;
-    if (int rc = check_dev_ptr(grad_dev, "grad_dev")) return rc;
+    if (int rc = check_dev_ptr(e, grad_dev, "grad_dev")) return rc;
     DeviceGuard guard(e->device);
     ga::Window w;
     int64_t tau = 0;
@@ -921,7 +956,7 @@ int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* cons
 
 int ga_get(ga_engine* e, int which, float* out_dev) {
     if (int rc = check_engine(e)) return rc;
-    if (int rc = check_dev_ptr(out_dev, "out_dev")) return rc;
+    if (int rc = check_dev_ptr(e, out_dev, "out_dev")) return rc;
     DeviceGuard guard(e->device);
     const float* src = which == GA_THETA ? e->theta : which == GA_V ? e->vel : which == GA_M ? e->mom : nullptr;
     if (which == GA_V2) {
@@ -945,7 +980,7 @@ int ga_get(ga_engine* e, int which, float* out_dev) {
 int ga_get_worker_momentum(ga_engine* e, int worker, float* out_dev) {
     if (int rc = check_engine(e)) return rc;
     if (int rc = check_worker(e, worker)) return rc;
-    if (int rc = check_dev_ptr(out_dev, "out_dev")) return rc;
+    if (int rc = check_dev_ptr(e, out_dev, "out_dev")) return rc;
     if (!e->is_dana()) return fail(GA_ERR_STATE, "only the DANA variants keep a momentum vector per worker");
     DeviceGuard guard(e->device);
     GA_CUDA(e, cudaMemcpyAsync(out_dev, e->vrow(worker), sizeof(float) * (size_t)e->d, cudaMemcpyDeviceToDevice, e->stream));
@@ -955,7 +990,7 @@ int ga_get_worker_momentum(ga_engine* e, int worker, float* out_dev) {
 int ga_gap(ga_engine* e, int worker, float* gap_out_dev) {
     if (int rc = check_engine(e)) return rc;
     if (int rc = check_worker(e, worker)) return rc;
-    if (int rc = check_dev_ptr(gap_out_dev, "gap_out_dev")) return rc;
+    if (int rc = check_dev_ptr(e, gap_out_dev, "gap_out_dev")) return rc;
     if (e->is_layer()) return fail(GA_ERR_STATE, "the layer-wise variant has one Gap per layer: see ga_get_layer_state");
     DeviceGuard guard(e->device);
     ga::ga_gap_kernel<<<grid_1d(e->d, 256, e->sms * 8), 256, 0, e->stream>>>(

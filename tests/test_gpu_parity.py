@@ -757,6 +757,20 @@ def test_bad_arguments_return_errors(P):
     assert l.ga_push_batch(h, sched, ptrs, -1, None) == P.GA_ERR_ARG
     assert eng.push(0, g) == 1 and eng.num_arrivals == 1     # still usable
     assert l.ga_set_option(h, P.GA_OPT_C_ORDER, 1.0) == P.GA_ERR_STATE
+    # ordinary host memory handed over as device memory is refused before any kernel could touch it
+    import numpy as np
+    host = np.zeros(1024 + 8, dtype=np.float32)
+    addr = (host.ctypes.data + 15) // 16 * 16
+    assert l.ga_push(h, 0, addr) == P.GA_ERR_ARG and "host memory" in P.last_error()
+    ptrs = (ctypes.c_void_p * 2)(g.data_ptr(), addr)
+    sched = (ctypes.c_int * 2)(0, 1)
+    assert l.ga_push_batch(h, sched, ptrs, 2, None) == P.GA_ERR_ARG and "gradient 1" in P.last_error()
+    assert l.ga_get(h, P.GA_THETA, addr) == P.GA_ERR_ARG
+    assert l.ga_set_params(h, addr) == P.GA_ERR_ARG
+    assert eng.num_arrivals == 1
+    pinned = torch.zeros(1000).pin_memory()                 # pinned host memory is reachable from the device
+    assert l.ga_push(h, 1, pinned.data_ptr()) == 2
+    assert torch.isfinite(eng.get(P.GA_THETA)).all()
     eng.close()
 
 
