@@ -209,7 +209,8 @@ int ga_push_batch(ga_engine* e, const int* schedule_host, const float* const* gr
  * schedule[j] after its arrival (n_params floats each). The parameter range is processed in
  * chunks so that host-to-device copies, the update kernel and device-to-host copies overlap,
  * across the windows of the call as well as within them. Synchronous: returns when all results
- * are in host memory. Allocates its staging buffers (2 x 16 x 16 MiB) on first use.
+ * are in host memory. Allocates its staging buffers (2 x 16 x 16 MiB) on first use. A buffer that
+ * is device memory is refused (GA_ERR_ARG, nothing applied); pageable host memory works, slower.
  * GA_GA_LAYER needs a whole gradient before a layer's norm is known: there the call stages whole
  * vectors, one arrival at a time (two staging buffers of n_params floats), the copy-in of the next
  * arrival and the copy-out of the previous one running beside the launches of the current. */

@@ -851,6 +851,17 @@ int ga_push_batch_host(ga_engine* e, const int* schedule_host, const float* cons
     if (sent_out_host)
         for (int j = 0; j < K; ++j)
             if (!sent_out_host[j]) return fail(GA_ERR_ARG, "sent_out_host[%d] is NULL", j);
+    // a device pointer where host memory is expected would make the copies fail half-way through the
+    // call: refuse it up front (the copies are whole vectors, so one query per buffer costs nothing)
+    for (int j = 0; j < K; ++j) {
+        for (const void* p : {(const void*)grads_host[j], (const void*)(sent_out_host ? sent_out_host[j] : nullptr)}) {
+            cudaPointerAttributes attr;
+            if (!p) continue;
+            if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) { cudaGetLastError(); continue; }
+            if (attr.type == cudaMemoryTypeDevice)
+                return fail(GA_ERR_ARG, "buffer %d of ga_push_batch_host is device memory; use ga_push_batch", j);
+        }
+    }
     DeviceGuard guard(e->device);
     if (int rc = ensure_host_path(e)) return rc;
     int launches = 0;

@@ -770,6 +770,13 @@ def test_bad_arguments_return_errors(P):
     assert eng.num_arrivals == 1
     pinned = torch.zeros(1000).pin_memory()                 # pinned host memory is reachable from the device
     assert l.ga_push(h, 1, pinned.data_ptr()) == 2
+    # and device memory where the host-buffer call expects host memory
+    hp = (ctypes.c_void_p * 1)(g.data_ptr())
+    one = (ctypes.c_int * 1)(2)
+    assert l.ga_push_batch_host(h, one, hp, 1, None, None) == P.GA_ERR_ARG and "device memory" in P.last_error()
+    assert eng.num_arrivals == 2
+    pageable = (ctypes.c_void_p * 1)(addr)                   # ordinary host memory is fine there
+    assert l.ga_push_batch_host(h, one, pageable, 1, None, None) >= 1 and eng.num_arrivals == 3
     assert torch.isfinite(eng.get(P.GA_THETA)).all()
     eng.close()
 
