@@ -55,6 +55,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-params", type=int, default=4_000_000)
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
+                    help="process group of the multi-rank arm (barrier and max over ranks only); gloo also lets "
+                         "more ranks than GPUs run, for checking that arm on a machine with one GPU")
     return ap.parse_args()
 
 
@@ -276,9 +279,15 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    n_dev = torch.cuda.device_count()
+    if world > 1 and args.backend == "nccl" and local_rank >= n_dev:
+        raise SystemExit(f"rank {rank}: no GPU {local_rank} (NCCL wants one GPU per rank)")
+    device_index = local_rank % n_dev          # gloo: ranks may share a GPU (their kernels never wait on one another)
+    torch.cuda.set_device(device_index)
+    if world > 1 and args.backend == "nccl":
+        dist.init_process_group("nccl", device_id=torch.device("cuda", device_index))
+    elif world > 1:
+        dist.init_process_group("gloo")
     P.lib()
 
     base = pick_workload(args)
@@ -305,7 +314,7 @@ def run_ours(args):
     for win in wins[:args.warmup]:
         run.step(win)
     barrier()
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(device_index)
     if rank == 0:
         sampler.start()
     events, launches0 = [], run.launches
@@ -358,6 +367,13 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = cpu_baseline_legs(base, args.variant, args.window, args.cpu_sample_params)
 
+    per_step_gb = alg_bytes / max(1, len(events)) / 1e9
+    state_mb = wl.d * 4 * (3 + wl.n_workers) / 1e6           # theta, v, m and the saved copies
+    if per_step_gb * 1e3 > 2 * 126 and state_mb > 2 * 126:
+        l2_note = f"inputs larger than L2 (each step streams {per_step_gb:.2f} GB; state {state_mb / 1e3:.1f} GB)"
+    else:
+        l2_note = (f"NOT larger than L2: each step streams {per_step_gb * 1e3:.0f} MB over a state of {state_mb:.0f} MB "
+                   "and L2 is not flushed between steps, so GB/s here is not a DRAM figure")
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -367,7 +383,7 @@ def run_ours(args):
                                    f"({wl.n_workers} saved copies), {args.variant}, window {args.window}, "
                                    f"{args.math} math",
                        "arrivals_timed": arrivals, "parallelism": f"range-sharded x{world}, no collective",
-                       "l2": "inputs larger than L2 (each step streams > 30 GB)",
+                       "l2": l2_note,
                        "timed": "CUDA events around each ga_push_batch call; gradient generation between "
                                 "steps is outside the events", "wall_s_incl_generation": wall},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,

@@ -68,3 +68,28 @@ def test_traffic_file_matches_the_kernel_source():
     else:
         assert value is None and "changed" in source
     assert bench.measured_traffic("SA", 16, "exact")[0] is None
+
+
+@pytest.mark.gpu
+def test_multi_rank_arm_runs_with_two_ranks_on_one_gpu():
+    """The N > 1 arm of bench.py (replicated schedule check, barrier, max over ranks, smaller
+    end-to-end leg) launched the way the contract says, with the gloo process group so that two ranks
+    can share the one GPU of a test box; their kernels never wait on one another."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+                          "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.join(ROOT, "bench.py"),
+                          "--gpus", "2", "--backend", "gloo", "--params", "300000", "--workers", "12", "--steps", "4",
+                          "--warmup", "3", "--e2e-steps", "1"],
+                         capture_output=True, text=True, cwd=ROOT, timeout=900)
+    assert out.returncode == 0, out.stderr[-3000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, out.stdout                      # rank 0 alone prints
+    j = json.loads(lines[0])
+    assert BASE_KEYS | {"roofline", "clocks"} <= set(j)
+    assert j["n_gpus"] == 2 and j["scaling"] == "weak" and j["value"] > 0 and j["gpu_launches"] == 4
+    assert j["cpu_baseline"] is None                         # the oracle is timed at N = 1 only
+    assert j["e2e"]["window"] == 2 and j["e2e"]["value"] > 0
+    assert "x2" in j["config"]["parallelism"] and "NOT larger than L2" in j["config"]["l2"]
