@@ -151,7 +151,9 @@ int ga_set_stream(ga_engine* e, void* cuda_stream);
 /* Learning rate eta_k for the arrivals that follow (decay, warm-up: Appendix "Hyperparameters").
  * eta_max of the C algorithm stays the rate given to ga_create (Algorithm "C Coefficient
  * Calculation" takes the maximal rate as an input, normally the first one), so the Gap penalty
- * relaxes as the rate decays (Section 5.1). lr must be positive and finite. */
+ * relaxes as the rate decays (Section 5.1). The momentum vector is kept free of the rate (v <- gamma
+ * v + g_hat, theta <- theta - eta_k v, as the master algorithms are printed), so a change of rate
+ * needs no correction of v. lr must be positive and finite. */
 int ga_set_lr(ga_engine* e, float lr);
 
 /* GA_GA_LAYER only, before the first arrival: layer p is elements [offsets_host[p],
